@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Benchmark of the PODS hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+pods_select -> pods_compact -> grpo_seq_weights -> grpo_loss_chunk per chunk -> grpo_loss_finalize.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line (rank 0).  `value` is kept tokens per second with every input resident in HBM;
+`e2e` is the same metric through the host-buffer entry point with the copies inside the timed region;
+`roofline` is the fused loss kernel against the measured HBM copy rate; `cpu_baseline` is the CPU
+checker timed on a bounded sample of the same rows.  With --gpus N > 1 (torchrun) every rank runs an
+independent replica of the batch (the path has no exchange step) and the rates add up.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2504_13818_b200 import workloads as wl  # noqa: E402
+
+METRIC = "kept-token GRPO loss+grad tokens/s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_qwen_vocab")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--select-bench", action="store_true", help="also time pods_select on configs 3 and 4")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        for line in self.file.read().splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                sm.append(float(p[0]))
+                smax.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+
+class Batch:
+    """Device-resident inputs of one step of workload `w`, and the buffers the step writes."""
+
+    def __init__(self, w, dev):
+        from paper_2504_13818_b200 import binding
+        self.w, self.dev, self.b = w, dev, binding
+        self.rewards_h = wl.make_rewards(w)
+        self.lengths_h, self.src_tokens_h = wl.make_rollouts(w)
+        self.rewards = torch.from_numpy(self.rewards_h).to(dev)
+        self.lengths = torch.from_numpy(self.lengths_h).to(dev)
+        self.src_tokens = torch.from_numpy(self.src_tokens_h).to(dev)
+        self.status = binding.new_status(dev)
+        self.M = w.G * w.m
+        # set-up pass (untimed): which rollouts are kept decides the rows the logits are drawn for
+        self.idx, self.adv, self.k = binding.pods_select(self.rewards, w.m, status=self.status)
+        cu, toks, _ = binding.pods_compact(self.idx, w.n, self.lengths, self.src_tokens, status=self.status)
+        self.T = int(cu[-1].item())
+        self.tokens0 = toks[: self.T].contiguous()
+        self.logits = wl.make_logits_device(w, self.tokens0)
+        lt = wl.library_logp(self.logits, self.tokens0).cpu().numpy()
+        old, ref = wl.make_old_ref(w, lt)
+        # old/ref log-probs live in rollout storage like the tokens, and are compacted with them
+        R, ld = self.src_tokens_h.shape
+        self.src_old_h = np.zeros((R, ld), np.float32)
+        self.src_ref_h = np.zeros((R, ld), np.float32)
+        cu_h, idx_h = cu.cpu().numpy(), self.idx.cpu().numpy()
+        for i in range(self.M):
+            g, j = divmod(i, w.m)
+            row = g * w.n + int(idx_h[g, j])
+            L = int(cu_h[i + 1] - cu_h[i])
+            self.src_old_h[row, :L] = old[cu_h[i]:cu_h[i + 1]]
+            self.src_ref_h[row, :L] = ref[cu_h[i]:cu_h[i + 1]]
+        self.src_old = torch.from_numpy(self.src_old_h).to(dev)
+        self.src_ref = torch.from_numpy(self.src_ref_h).to(dev)
+        # outputs / scratch, allocated once
+        T = self.T
+        self.cu = torch.empty(self.M + 1, dtype=torch.int64, device=dev)
+        self.tokens = torch.empty(T, dtype=torch.int32, device=dev)
+        self.old = torch.empty(T, dtype=torch.float32, device=dev)
+        self.ref = torch.empty(T, dtype=torch.float32, device=dev)
+        self.dlogits = torch.empty_like(self.logits)
+        self.logp = torch.empty(T, dtype=torch.float32, device=dev)
+        self.loss = torch.empty(1, dtype=torch.float32, device=dev)
+        self.loss_acc = torch.zeros(1, dtype=torch.float64, device=dev)
+        self.seq_weight = torch.empty(self.M, dtype=torch.float64, device=dev)
+        self.chunk = min(w.chunk_rows, T)
+        self.ws = torch.empty(binding.grpo_loss_chunk_workspace_bytes(self.chunk), dtype=torch.uint8, device=dev)
+        self.n_chunks = (T + self.chunk - 1) // self.chunk
+        self.launches_per_step = 1 + 2 + 1 + 1 + 2 * self.n_chunks + 1   # select, compact(2), zero, weights, chunks, finalize
+        self.loss_events = []
+
+    def step(self, record=False):
+        b, w = self.b, self.w
+        b.pods_select_into(self.rewards, w.m, self.idx, self.adv, self.k, status=self.status)
+        b.pods_compact(self.idx, w.n, self.lengths, self.src_tokens, [self.src_old, self.src_ref], T_cap=self.T,
+                       status=self.status, out=(self.cu, self.tokens, [self.old, self.ref]))
+        self.loss_acc.zero_()
+        b.grpo_seq_weights(None, self.cu, out=self.seq_weight)
+        for c in range(self.n_chunks):
+            lo = c * self.chunk
+            hi = min(self.T, lo + self.chunk)
+            if record:
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+            b.grpo_loss_chunk(self.logits[lo:hi], self.tokens[lo:hi], self.old[lo:hi], self.ref[lo:hi], self.adv,
+                              self.seq_weight, self.cu, lo, None, w.eps, w.beta, self.loss_acc, self.logp[lo:hi],
+                              self.dlogits[lo:hi], self.ws, status=self.status)
+            if record:
+                e1.record()
+                self.loss_events.append((e0, e1, hi - lo))
+        b.grpo_loss_finalize(self.loss_acc, self.loss)
+
+
+def time_select(name, dev, steps, warmup):
+    """pods_select alone on a selection-only workload, L2 flushed between launches."""
+    from paper_2504_13818_b200 import binding
+    w = wl.WORKLOADS[name]
+    r = torch.from_numpy(wl.make_rewards(w)).to(dev)
+    idx = torch.empty((w.G, w.m), dtype=torch.int32, device=dev)
+    adv = torch.empty((w.G, w.m), dtype=torch.float32, device=dev)
+    k = torch.empty(w.G, dtype=torch.int32, device=dev)
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    times = []
+    for i in range(warmup + steps):
+        flush.fill_(i & 0xff)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        binding.pods_select_into(r, w.m, idx, adv, k)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            times.append(e0.elapsed_time(e1))
+    ms = statistics.median(times)
+    bytes_alg = w.G * (4 * w.n + 8 * w.m + 4)
+    peak, _ = measured_peak()
+    return {"workload": name, "G": w.G, "n": w.n, "m": w.m, "ms": ms, "groups_per_s": w.G / (ms * 1e-3),
+            "GBps": bytes_alg / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": bytes_alg / (ms * 1e-3) / 1e9 / peak}
+
+
+def cpu_baseline(batch, budget_rows=None):
+    """The CPU checker, as it stands, on a bounded sample of the same batch (rank 0, N=1 only)."""
+    import oracle
+    w = batch.w
+    t0 = time.perf_counter()
+    sel = oracle.select(batch.rewards_h, w.m)
+    cu, toks, _, seq_of_row = oracle.compact(sel["idx"], w.n, batch.lengths_h, batch.src_tokens_h)
+    t_sel = time.perf_counter() - t0
+    T = int(cu[-1])
+    cores = oracle.num_threads()
+    rows = budget_rows or max(cores, min(T, 192 * cores if w.V > 50000 else 20000))
+    rows = min(rows, T)
+    lg = batch.logits[:rows].view(torch.uint16).cpu().numpy()
+    old = batch.old[:rows].cpu().numpy()
+    ref = batch.ref[:rows].cpu().numpy()
+    mask = np.ones(T, np.uint8)
+    t0 = time.perf_counter()
+    sw = oracle.seq_weights(mask, cu)
+    out = oracle.grpo_rows(lg, toks[:rows], old, ref, sel["adv"].astype(np.float32).reshape(-1), sw,
+                           seq_of_row[:rows], mask[:rows], w.eps, w.beta, want_dlogits=True)
+    t_rows = time.perf_counter() - t0
+    del out
+    # selection and compaction are done in full, the loss on `rows` of T rows: scale to a whole step
+    step_s = t_sel + t_rows * (T / rows)
+    return {"value": T / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "select+compact in full (%d groups), loss+grad on the first %d of %d rows (V=%d), "
+                      "extrapolated to the step" % (w.G, rows, T, w.V),
+            "seconds_measured": t_sel + t_rows}
+
+
+def run_ours(args):
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2504_13818_b200 import binding
+    binding.load()
+    w = wl.WORKLOADS[args.workload]
+    batch = Batch(w, dev)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        batch.step()
+    torch.cuda.synchronize()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        batch.step(record=True)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    status = binding.read_status(batch.status)
+
+    # the dominant kernel: the fused loss rows kernel, timed per chunk launch on its own stream
+    full = [(a.elapsed_time(b_), rows) for a, b_, rows in batch.loss_events if rows == batch.chunk]
+    per_launch_ms = statistics.mean(t for t, _ in full)
+    bytes_per_token = 4 * w.V + 21
+    achieved = bytes_per_token * batch.chunk / (per_launch_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    roofline = {"kernel": "grpo_loss_rows_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
+                "frac_of_nominal_8TBps": achieved / 8000.0, "traffic": None,
+                "bytes_per_launch": bytes_per_token * batch.chunk, "ms_per_launch": per_launch_ms,
+                "rows_per_launch": batch.chunk}
+
+    out = {
+        "metric": METRIC, "value": world * batch.T * args.steps / (ms_total * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 logits, f32 exp, f64 scalars",
+        "data": "synthetic",
+        "config": {"workload": w.name, "G": w.G, "n": w.n, "m": w.m, "V": w.V, "kept_tokens": batch.T,
+                   "chunk_rows": batch.chunk, "l2": "inputs larger than L2 (logits %.1f GB per step)"
+                   % (batch.T * w.V * 2 / 1e9), "replicas": world},
+        "gpu_launches": batch.launches_per_step * args.steps,
+        "device_status_word": status,
+        "loss": float(batch.loss.item()),
+        "roofline": roofline,
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_e2e:
+        out["e2e"] = run_e2e(batch, args)
+    else:
+        out["e2e"] = None
+    if rank == 0 and world == 1 and args.select_bench:
+        out["pods_select"] = [time_select(nm, dev, 20, 3) for nm in ("c3_select_mixed", "c4_select_ties")]
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(batch)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_e2e(batch, args):
+    """The same step through the host-buffer entry point: inputs in pinned host memory, results read back."""
+    from paper_2504_13818_b200 import binding
+    if not hasattr(binding, "pods_step_host"):
+        return None
+    return binding_e2e(batch, args)
+
+
+def binding_e2e(batch, args):
+    from paper_2504_13818_b200 import binding
+    w = batch.w
+    host = binding.HostStep(w.G, w.n, w.m, batch.src_tokens_h.shape[1], batch.T, w.V, chunk_rows=2048)
+    host.set_inputs(batch.rewards_h, batch.lengths_h, batch.src_tokens_h, batch.src_old_h, batch.src_ref_h,
+                    batch.logits)
+    steps = max(2, min(args.steps, 3))
+    for _ in range(1):
+        host.run(w.eps, w.beta)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        host.run(w.eps, w.beta)
+    dt = time.perf_counter() - t0
+    return {"value": batch.T * steps / dt, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes,
+            "d2h_bytes_per_step": host.d2h_bytes, "steps": steps, "ms_per_step": dt / steps * 1e3,
+            "loss": host.loss()}
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the CPU checker on the host cores
+# --------------------------------------------------------------------------------------------
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    w = wl.WORKLOADS[args.workload]
+    rewards = wl.make_rewards(w)
+    lengths, src_tokens = wl.make_rollouts(w)
+    sel = oracle.select(rewards, w.m)
+    cu, toks, _, seq_of_row = oracle.compact(sel["idx"], w.n, lengths, src_tokens)
+    T = int(cu[-1])
+    cores = oracle.num_threads()
+    rows = min(T, 48 * cores if w.V > 50000 else 4096)
+    sub = wl.shrink_rows(w, rows) if hasattr(wl, "shrink_rows") else w
+    logits = wl.make_logits_host(sub, toks[:rows])
+    old, ref = wl.make_old_ref(w, wl.host_logp_tilde(logits, toks[:rows]))
+    mask = np.ones(T, np.uint8)
+    adv32 = sel["adv"].astype(np.float32).reshape(-1)
+
+    def step():
+        s = oracle.select(rewards, w.m)
+        c, tk, _, sor = oracle.compact(s["idx"], w.n, lengths, src_tokens)
+        sw = oracle.seq_weights(mask, c)
+        o = oracle.grpo_rows(logits, tk[:rows], old, ref, adv32, sw, sor[:rows], mask[:rows], w.eps, w.beta)
+        return o
+
+    for _ in range(max(1, min(args.warmup, 1))):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = rows * args.steps / dt
+    sample = "each step: select+compact in full (%d groups) and loss+grad on %d of %d rows (V=%d)" % (w.G, rows, T, w.V)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "G": w.G, "n": w.n, "m": w.m, "V": w.V, "kept_tokens": T, "rows_per_step": rows},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,165 @@
+/*
+ * pods.h - C ABI of the B200 (sm_100a) hot path of PODS, "Policy Optimization with
+ * Down-Sampling" (arxiv 2504.13818): per prompt group, max-variance down-sampling of n
+ * rollout rewards to m rollouts, GRPO advantages on the kept subset, concatenation of the
+ * kept rollouts, and the GRPO-PODS token objective with its gradient w.r.t. the logits.
+ *
+ * Conventions for every call
+ *   - Pointers marked [dev] are device pointers on the current CUDA device, [host] are host
+ *     pointers.  The caller owns every buffer; the library allocates no device memory and
+ *     keeps no state between calls (except pods_step_host, which says what it allocates).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work and return; outputs are valid once the stream has reached that point.
+ *   - The return value is a pods_status.  Errors that the host can see (sizes, null or
+ *     misaligned pointers, workspace too small) are returned before anything is launched.
+ *   - Anomalies only the device can see (non-finite reward, token id outside [0,V), packed
+ *     output capacity exceeded) OR a bit into *status [dev, uint32, may be NULL, never
+ *     cleared by the library] and the kernel carries on with a defined substitute.  No kernel
+ *     traps or waits without bound.
+ *   - Notation follows the paper: G prompt groups, n rollouts per group, m kept per group,
+ *     M = G*m kept rollouts, T kept tokens, V vocabulary size, |o_i| tokens of rollout i.
+ */
+#ifndef PODS_H_
+#define PODS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PODS_OK = 0,
+    PODS_ERR_INVALID_ARG = 1,   /* bad size, null pointer, misaligned pointer */
+    PODS_ERR_UNSUPPORTED = 2,   /* n above PODS_MAX_N, unknown rule */
+    PODS_ERR_WORKSPACE = 3,     /* workspace missing or too small */
+    PODS_ERR_CUDA = 4           /* a CUDA runtime call failed (launch, copy) */
+} pods_status;
+
+/* Bits of the device status word. */
+#define PODS_STATUS_NONFINITE_REWARD 0x1u  /* a reward was NaN or +-inf (sorted as NaN > +inf > finite) */
+#define PODS_STATUS_TOKEN_RANGE      0x2u  /* a token id was outside [0,V); token 0 was used instead      */
+#define PODS_STATUS_CAPACITY         0x4u  /* pods_compact: T exceeded T_cap (the excess was not written),
+                                              or a length exceeded src_ld (it was cut to src_ld)          */
+#define PODS_STATUS_NEG_LENGTH       0x8u  /* pods_compact: a negative length was treated as 0            */
+
+/* Down-sampling rules D(o, r; m) of Section 3.2 / 3.3. */
+typedef enum {
+    PODS_RULE_MAXVAR = 0,      /* max-variance down-sampling, Section 3.3, Algorithm 2 */
+    PODS_RULE_MAXREWARD = 1,   /* the m highest rewards, Section 3.2                   */
+    PODS_RULE_RANDOM = 2,      /* uniform m-subset, Section 3.2                        */
+    PODS_RULE_PERCENTILE = 3   /* the (j+0.5)/m quantiles, Section 3.2                 */
+} pods_rule;
+
+#define PODS_FLAG_ADV_BEFORE 0x1u  /* advantages from full-group statistics (Appendix A.3 "Before") */
+#define PODS_FLAG_STD_SAMPLE 0x2u  /* divide by (count-1) instead of count in the standard deviation  */
+
+#define PODS_MAX_N 1024            /* largest supported group size n */
+
+const char* pods_version(void);
+const char* pods_status_string(int status);
+
+/* Copy the device status word to *host_value [host]; synchronises `stream`. */
+int pods_read_status(const uint32_t* status /*dev*/, uint32_t* host_value /*host*/, void* stream);
+
+/*
+ * pods_select - down-sampling rule D(o, r; m) -> S (Definition 3.1) for G groups at once, and
+ * the advantages a_{S,i} = (r_i - mu_S) / sigma_S of Section 3.2.
+ *
+ * PODS_RULE_MAXVAR is Algorithm 2 with the prefix sums of Theorem 1's proof: argsort the
+ * rewards (ties by index, -0 == +0), and over k = 0..m take the k highest and m-k lowest whose
+ * variance is largest, the smallest such k on ties (Algorithm 2 replaces only on a strictly
+ * larger variance).  Split scores are evaluated in fp64 on rewards centred on the group minimum.
+ * PODS_RULE_RANDOM keeps the m rollouts with the smallest 32-bit Philox4x32-10 words (counter
+ * (i, 0, g lo, g hi), key = seed, first output word; ties by index).  PODS_RULE_PERCENTILE keeps
+ * sorted positions floor((j+0.5) n/m), j = 0..m-1.
+ *
+ *   rewards [dev] fp32 [G,n] row-major            idx   [dev] int32 [G,m], ascending original index
+ *   adv     [dev] fp32 [G,m] aligned with idx     k_out [dev] int32 [G] or NULL: highest-reward count k
+ *                                                       (m for MAXREWARD, -1 for RANDOM/PERCENTILE)
+ * sigma_S is the population (divide by m) standard deviation unless PODS_FLAG_STD_SAMPLE; if it
+ * is 0 every advantage of the group is 0.  Requires 1 <= m <= n <= PODS_MAX_N, G >= 0.
+ */
+int pods_select(const float* rewards, int64_t G, int32_t n, int32_t m, int32_t rule, uint64_t seed,
+                uint32_t flags, int32_t* idx, float* adv, int32_t* k_out, uint32_t* status, void* stream);
+
+/*
+ * pods_compact - "apply the same procedure to each prompt and then concatenate the down-sampled
+ * rollouts" (text after Algorithm 1).  Rollout j of group g is row g*n+j of the padded storage;
+ * kept rollout number i = g*m+j' is rollout idx[g,j'].
+ *
+ *   idx        [dev] int32 [G,m]                   lengths   [dev] int32 [G*n] tokens per rollout
+ *   src_tokens [dev] int32 [G*n, src_ld]           src_f32   [host] array of n_f32 (<= 4) [dev] fp32
+ *   dst_tokens [dev] int32 [T_cap]                            [G*n, src_ld] per-token streams (or NULL)
+ *   dst_f32    [host] array of n_f32 [dev] fp32 [T_cap]
+ *   cu_seqlens [dev] int64 [M+1]: exclusive prefix sums of the kept lengths; cu_seqlens[M] = T
+ * Tokens beyond T_cap are not written and PODS_STATUS_CAPACITY is raised.
+ */
+int pods_compact(const int32_t* idx, int64_t G, int32_t n, int32_t m, const int32_t* lengths,
+                 const int32_t* src_tokens, int64_t src_ld, const float* const* src_f32, int32_t n_f32,
+                 int64_t* cu_seqlens, int32_t* dst_tokens, float* const* dst_f32, int64_t T_cap,
+                 uint32_t* status, void* stream);
+
+/*
+ * grpo_seq_weights - the factor 1/(M |o_i|) in front of the token sum of L_PODS (Section 3.2; the
+ * 1/m of one prompt becomes 1/M over the concatenated batch).  |o_i| counts tokens with mask != 0
+ * (all tokens if mask is NULL); an empty rollout gets weight 0.
+ *   mask [dev] uint8 [T] or NULL    cu_seqlens [dev] int64 [M+1]    seq_weight [dev] fp64 [M]
+ */
+int grpo_seq_weights(const uint8_t* mask, const int64_t* cu_seqlens, int64_t M, double* seq_weight, void* stream);
+
+/* Bytes of workspace grpo_loss_chunk needs for a chunk of T_chunk rows. */
+size_t grpo_loss_chunk_workspace_bytes(int64_t T_chunk);
+
+/*
+ * grpo_loss_chunk - the token terms of L_PODS(theta, S) (Section 3.2) and d loss / d logits for
+ * rows [row0, row0 + T_chunk) of the packed kept tokens, in one kernel.  Per row t of rollout i:
+ *   logp = log softmax(logits[t,:])[token]        rho = exp(logp - old_logp)
+ *   loss_t = -min(rho a_i, clip(rho, 1-eps, 1+eps) a_i) + beta (exp(d) - d - 1),  d = ref_logp - logp
+ *   g_t = grad_scale mask_t w_i (-a_i rho [rho a_i <= clip(rho) a_i] + beta (1 - exp(d)))
+ *   dlogits[t,v] = g_t ([v == token] - softmax(logits[t,:])[v])   rounded to bf16 (nearest even)
+ * and sum_t mask_t w_i loss_t is ADDED to *loss_acc (the caller zeroes it before the first chunk;
+ * the loss is minimised, i.e. it is minus the paper's objective, plus the KL penalty whose
+ * coefficient is Table 2's "KL Coefficient").  Rows with mask 0 get logp but a zero dlogits row.
+ *
+ *   logits  [dev] bf16 [T_chunk, V], row pitch ldl elements.  Fast path: 16-byte aligned base and
+ *           ldl % 8 == 0; anything else takes a slower element-wise path.
+ *   tokens, old_logp, ref_logp (NULL allowed iff beta == 0), mask (NULL = all ones), logp:
+ *           [dev] arrays of T_chunk entries for this chunk's rows (int32, fp32, fp32, uint8, fp32 out)
+ *   adv [dev] fp32 [M]; seq_weight [dev] fp64 [M]; cu_seqlens [dev] int64 [M+1]: row0 + t is mapped
+ *           to its rollout through cu_seqlens
+ *   dlogits [dev] bf16 [T_chunk, V] pitch ldd; may be the same buffer as logits (in place, ldd == ldl),
+ *           must not overlap it otherwise
+ *   loss_acc [dev] fp64 scalar; workspace [dev] of grpo_loss_chunk_workspace_bytes(T_chunk), 16-byte aligned
+ */
+int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
+                    const float* ref_logp, const float* adv, const double* seq_weight,
+                    const int64_t* cu_seqlens, int64_t M, int64_t row0, const uint8_t* mask, int64_t T_chunk,
+                    int32_t V, float eps, float beta, float grad_scale, double* loss_acc, float* logp,
+                    void* dlogits, int64_t ldd, void* workspace, size_t workspace_bytes, uint32_t* status,
+                    void* stream);
+
+/* Bytes of workspace grpo_loss_fwd_bwd needs. */
+size_t grpo_loss_workspace_bytes(int64_t T, int64_t M, int64_t chunk_rows);
+
+/*
+ * grpo_loss_fwd_bwd - L_PODS(theta, S) over the whole packed batch (Section 3.2):
+ *   (logits, tokens, old_logp, ref_logp, adv, mask, eps, beta) -> loss, logp, dlogits.
+ * Computes the rollout weights, runs grpo_loss_chunk over chunks of chunk_rows rows (<= 0: one
+ * chunk) and writes loss [dev] fp32 scalar = (1/M) sum_i (1/|o_i|) sum_t mask_t loss_t.
+ * Arguments as in grpo_loss_chunk, with per-token arrays of T entries.
+ */
+int grpo_loss_fwd_bwd(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
+                      const float* ref_logp, const float* adv, const int64_t* cu_seqlens, int64_t M,
+                      const uint8_t* mask, int64_t T, int32_t V, float eps, float beta, int64_t chunk_rows,
+                      float* loss, float* logp, void* dlogits, int64_t ldd, void* workspace,
+                      size_t workspace_bytes, uint32_t* status, void* stream);
+
+/* Convert the fp64 accumulator of grpo_loss_chunk calls to the fp32 loss.  Both [dev]. */
+int grpo_loss_finalize(const double* loss_acc, float* loss, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PODS_H_ */

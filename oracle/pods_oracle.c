@@ -78,13 +78,13 @@ void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* ou
     philox4x32_10(ctr, key, out);
 }
 
-/* 64 random bits for rollout i of group g under a seed. */
+/* The random word of rollout i of group g under a seed: the first output word. */
 static uint64_t random_key(uint64_t seed, int64_t g, int32_t i) {
     uint32_t ctr[4] = {(uint32_t)i, 0u, (uint32_t)((uint64_t)g & 0xffffffffu), (uint32_t)((uint64_t)g >> 32)};
     uint32_t key[2] = {(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32)};
     uint32_t out[4];
     philox4x32_10(ctr, key, out);
-    return ((uint64_t)out[1] << 32) | out[0];
+    return (uint64_t)out[0];
 }
 
 /* ------------------------------------------------------------------------- */
@@ -149,7 +149,8 @@ int oracle_select(const float* rewards, int64_t G, int32_t n, int32_t m, int32_t
         double rel_gap = INFINITY;
 
         if (rule == RULE_RANDOM) {
-            /* D_rand: a uniformly random m-subset = the m smallest of n i.i.d. keys. */
+            /* D_rand: a uniformly random m-subset = the m smallest of n i.i.d. 32-bit words
+             * (equal words, probability ~n^2 2^-33 per group, fall back to index order). */
             key_index* ki = (key_index*)malloc(sizeof(key_index) * (size_t)n);
             for (int i = 0; i < n; ++i) { ki[i].u = random_key(seed, g, i); ki[i].i = i; }
             qsort(ki, (size_t)n, sizeof(key_index), cmp_key_index);
@@ -321,6 +322,11 @@ int64_t oracle_grpo_rows(const uint16_t* logits, int64_t ldl, int64_t T, int32_t
         grpo_row(x, V, tok, (double)old_logp[t], ref_logp ? (double)ref_logp[t] : 0.0, ref_logp != NULL,
                  (double)adv[i], (double)eps, (double)beta, w, &lp, &el, &dl, &mg,
                  dlogits ? dlogits + t * (int64_t)V : NULL);
+        if (!mask[t] || w == 0.0) {
+            /* not a token of any rollout's sum: no gradient, whatever old/ref hold there */
+            dl = 0.0;
+            if (dlogits) memset(dlogits + t * (int64_t)V, 0, sizeof(double) * (size_t)V);
+        }
         if (logp) logp[t] = lp;
         if (ell) ell[t] = el;
         if (g) g[t] = w * dl;
@@ -342,6 +348,10 @@ void oracle_grpo_rows_f64(const double* logits, int64_t T, int32_t V, const int3
         grpo_row(logits + t * (int64_t)V, V, tokens[t], old_logp[t], ref_logp ? ref_logp[t] : 0.0,
                  ref_logp != NULL, adv[i], eps, beta, w, &lp, &el, &dl, &mg,
                  dlogits ? dlogits + t * (int64_t)V : NULL);
+        if (!mask[t] || w == 0.0) {
+            dl = 0.0;
+            if (dlogits) memset(dlogits + t * (int64_t)V, 0, sizeof(double) * (size_t)V);
+        }
         if (logp) logp[t] = lp;
         if (ell) ell[t] = el;
         if (g) g[t] = w * dl;

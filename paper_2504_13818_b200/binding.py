@@ -1,0 +1,238 @@
+"""ctypes binding of the C-ABI CUDA library declared in ``include/pods.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (torch is used for device
+memory and streams), checks dtypes/contiguity, passes raw pointers and sizes to the library
+call of the same name on the current stream, and raises on a non-zero status.  All computation
+happens in the library's kernels; there is no CPU or eager fallback, and a missing library is
+an error.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpods_b200.so")
+
+RULE_MAXVAR, RULE_MAXREWARD, RULE_RANDOM, RULE_PERCENTILE = 0, 1, 2, 3
+FLAG_ADV_BEFORE, FLAG_STD_SAMPLE = 1, 2
+STATUS_NONFINITE_REWARD, STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_NEG_LENGTH = 1, 2, 4, 8
+MAX_N = 1024
+
+# name -> (restype, argtypes); mirrors include/pods.h
+_p, _i64, _i32, _u64, _u32, _f32, _sz = (C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_uint32,
+                                         C.c_float, C.c_size_t)
+SIGNATURES = {
+    "pods_version": (C.c_char_p, []),
+    "pods_status_string": (C.c_char_p, [C.c_int]),
+    "pods_read_status": (C.c_int, [_p, _p, _p]),
+    "pods_select": (C.c_int, [_p, _i64, _i32, _i32, _i32, _u64, _u32, _p, _p, _p, _p, _p]),
+    "pods_compact": (C.c_int, [_p, _i64, _i32, _i32, _p, _p, _i64, _p, _i32, _p, _p, _p, _i64, _p, _p]),
+    "grpo_seq_weights": (C.c_int, [_p, _p, _i64, _p, _p]),
+    "grpo_loss_chunk_workspace_bytes": (_sz, [_i64]),
+    "grpo_loss_chunk": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _p, _i64, _i64, _p, _i64, _i32, _f32, _f32,
+                                  _f32, _p, _p, _p, _i64, _p, _sz, _p, _p]),
+    "grpo_loss_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "grpo_loss_fwd_bwd": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i32, _f32, _f32, _i64,
+                                    _p, _p, _p, _i64, _p, _sz, _p, _p]),
+    "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
+}
+
+_lib = None
+
+
+class PodsError(RuntimeError):
+    pass
+
+
+def load():
+    """Load libpods_b200.so (built in-tree by csrc/build.py).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise PodsError("CUDA library %s is missing: run `python -m paper_2504_13818_b200.csrc.build` "
+                        "(there is no CPU fallback)" % LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise PodsError("%s failed: %s (status %d)" % (what, load().pods_status_string(rc).decode(), rc))
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t, dtype, name, optional=False):
+    if t is None:
+        if optional:
+            return None
+        raise PodsError("%s is required" % name)
+    if not (isinstance(t, torch.Tensor) and t.is_cuda):
+        raise PodsError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype:
+        raise PodsError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise PodsError("%s must be contiguous" % name)
+    return C.c_void_p(t.data_ptr())
+
+
+def _rows(t, name):
+    """Pointer and row pitch of a 2-D bf16 tensor whose rows are contiguous."""
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 2):
+        raise PodsError("%s must be a 2-D CUDA bfloat16 tensor" % name)
+    if t.stride(1) != 1:
+        raise PodsError("%s rows must be contiguous" % name)
+    return C.c_void_p(t.data_ptr()), (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1]))
+
+
+def version() -> str:
+    return load().pods_version().decode()
+
+
+def new_status(device=None):
+    return torch.zeros(1, dtype=torch.int32, device=device or "cuda")
+
+
+def read_status(status) -> int:
+    out = C.c_uint32(0)
+    _check(load().pods_read_status(_dev(status, torch.int32, "status"), C.byref(out), _stream()), "pods_read_status")
+    return int(out.value)
+
+
+def pods_select(rewards, m, rule=RULE_MAXVAR, seed=0, flags=0, status=None, want_k=True):
+    """rewards [G,n] fp32 -> (idx [G,m] int32, adv [G,m] fp32, k [G] int32 or None)."""
+    rp = _dev(rewards, torch.float32, "rewards")
+    if rewards.dim() != 2:
+        raise PodsError("rewards must be [G,n]")
+    G, n = rewards.shape
+    idx = torch.empty((G, m), dtype=torch.int32, device=rewards.device)
+    adv = torch.empty((G, m), dtype=torch.float32, device=rewards.device)
+    k = torch.empty((G,), dtype=torch.int32, device=rewards.device) if want_k else None
+    rc = load().pods_select(rp, G, n, m, rule, seed, flags, C.c_void_p(idx.data_ptr()), C.c_void_p(adv.data_ptr()),
+                            C.c_void_p(k.data_ptr()) if want_k else None,
+                            _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "pods_select")
+    return idx, adv, k
+
+
+def pods_select_into(rewards, m, idx, adv, k=None, rule=RULE_MAXVAR, seed=0, flags=0, status=None):
+    """As pods_select with caller-provided outputs (no allocation)."""
+    G, n = rewards.shape
+    rc = load().pods_select(_dev(rewards, torch.float32, "rewards"), G, n, m, rule, seed, flags,
+                            _dev(idx, torch.int32, "idx"), _dev(adv, torch.float32, "adv"),
+                            _dev(k, torch.int32, "k", True), _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "pods_select")
+
+
+def pods_compact(idx, n, lengths, src_tokens, src_f32=(), T_cap=None, status=None, out=None):
+    """Pack the kept rollouts.  Returns (cu_seqlens int64 [M+1], tokens int32 [T_cap], [fp32 streams]).
+
+    ``T_cap`` defaults to M * src_ld (always enough).  ``out`` may carry pre-allocated
+    (cu_seqlens, tokens, [streams]) to write into.
+    """
+    G, m = idx.shape
+    src_ld = src_tokens.shape[1]
+    M = G * m
+    if T_cap is None:
+        T_cap = M * src_ld
+    dev = idx.device
+    if out is None:
+        cu = torch.empty(M + 1, dtype=torch.int64, device=dev)
+        toks = torch.empty(T_cap, dtype=torch.int32, device=dev)
+        dst = [torch.empty(T_cap, dtype=torch.float32, device=dev) for _ in src_f32]
+    else:
+        cu, toks, dst = out
+    k = len(src_f32)
+    src_arr = (C.c_void_p * max(k, 1))(*[_dev(s, torch.float32, "src_f32").value for s in src_f32])
+    dst_arr = (C.c_void_p * max(k, 1))(*[_dev(d, torch.float32, "dst_f32").value for d in dst])
+    for s in src_f32:
+        if tuple(s.shape) != tuple(src_tokens.shape):
+            raise PodsError("src_f32 streams must have the shape of src_tokens")
+    rc = load().pods_compact(_dev(idx, torch.int32, "idx"), G, n, m, _dev(lengths, torch.int32, "lengths"),
+                             _dev(src_tokens, torch.int32, "src_tokens"), src_ld,
+                             C.cast(src_arr, C.c_void_p) if k else None, k,
+                             _dev(cu, torch.int64, "cu_seqlens"), _dev(toks, torch.int32, "dst_tokens"),
+                             C.cast(dst_arr, C.c_void_p) if k else None, T_cap,
+                             _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "pods_compact")
+    return cu, toks, dst
+
+
+def grpo_seq_weights(mask, cu_seqlens, out=None):
+    M = cu_seqlens.shape[0] - 1
+    w = out if out is not None else torch.empty(M, dtype=torch.float64, device=cu_seqlens.device)
+    rc = load().grpo_seq_weights(_dev(mask, torch.uint8, "mask", True), _dev(cu_seqlens, torch.int64, "cu_seqlens"),
+                                 M, _dev(w, torch.float64, "seq_weight"), _stream())
+    _check(rc, "grpo_seq_weights")
+    return w
+
+
+def grpo_loss_chunk_workspace_bytes(T_chunk) -> int:
+    return int(load().grpo_loss_chunk_workspace_bytes(T_chunk))
+
+
+def grpo_loss_workspace_bytes(T, M, chunk_rows=0) -> int:
+    return int(load().grpo_loss_workspace_bytes(T, M, chunk_rows))
+
+
+def grpo_loss_chunk(logits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, row0, mask, eps, beta,
+                    loss_acc, logp, dlogits, workspace, grad_scale=1.0, status=None):
+    """One chunk of rows [row0, row0+T_chunk).  Per-token tensors hold this chunk's rows only."""
+    lp, ldl = _rows(logits, "logits")
+    dp, ldd = _rows(dlogits, "dlogits")
+    T, V = logits.shape
+    rc = load().grpo_loss_chunk(lp, ldl, _dev(tokens, torch.int32, "tokens"), _dev(old_logp, torch.float32, "old_logp"),
+                                _dev(ref_logp, torch.float32, "ref_logp", True), _dev(adv.reshape(-1), torch.float32, "adv"),
+                                _dev(seq_weight, torch.float64, "seq_weight"), _dev(cu_seqlens, torch.int64, "cu_seqlens"),
+                                cu_seqlens.shape[0] - 1, row0, _dev(mask, torch.uint8, "mask", True), T, V,
+                                eps, beta, grad_scale, _dev(loss_acc, torch.float64, "loss_acc"),
+                                _dev(logp, torch.float32, "logp"), dp, ldd,
+                                _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+                                _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "grpo_loss_chunk")
+
+
+def grpo_loss_finalize(loss_acc, loss):
+    _check(load().grpo_loss_finalize(_dev(loss_acc, torch.float64, "loss_acc"), _dev(loss, torch.float32, "loss"),
+                                     _stream()), "grpo_loss_finalize")
+
+
+def grpo_loss_fwd_bwd(logits, tokens, old_logp, ref_logp, adv, mask, eps, beta, cu_seqlens, chunk_rows=0,
+                      dlogits=None, logp=None, loss=None, workspace=None, status=None):
+    """(logits, tokens, old_logp, ref_logp, adv, mask, eps, beta) -> (loss [1] fp32, logp [T] fp32, dlogits).
+
+    ``dlogits`` may be ``logits`` itself (in place).  Missing outputs / workspace are allocated here.
+    """
+    T, V = logits.shape
+    M = cu_seqlens.shape[0] - 1
+    dev = logits.device
+    if dlogits is None:
+        dlogits = torch.empty_like(logits)
+    if logp is None:
+        logp = torch.empty(T, dtype=torch.float32, device=dev)
+    if loss is None:
+        loss = torch.empty(1, dtype=torch.float32, device=dev)
+    need = grpo_loss_workspace_bytes(T, M, chunk_rows)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    lp, ldl = _rows(logits, "logits")
+    dp, ldd = _rows(dlogits, "dlogits")
+    rc = load().grpo_loss_fwd_bwd(lp, ldl, _dev(tokens, torch.int32, "tokens"), _dev(old_logp, torch.float32, "old_logp"),
+                                  _dev(ref_logp, torch.float32, "ref_logp", True),
+                                  _dev(adv.reshape(-1), torch.float32, "adv"),
+                                  _dev(cu_seqlens, torch.int64, "cu_seqlens"), M,
+                                  _dev(mask, torch.uint8, "mask", True), T, V, eps, beta, chunk_rows,
+                                  _dev(loss, torch.float32, "loss"), _dev(logp, torch.float32, "logp"), dp, ldd,
+                                  _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+                                  _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "grpo_loss_fwd_bwd")
+    return loss, logp, dlogits

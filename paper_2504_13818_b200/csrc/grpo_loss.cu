@@ -1,0 +1,425 @@
+// grpo_loss: the GRPO-PODS token objective L_PODS(theta, S) of Section 3.2 and its gradient with
+// respect to the bf16 logits, fused: per row one streaming pass for the softmax statistics and the
+// target log-prob, the scalar loss terms, then the gradient row.
+//
+// Row kernel (one CTA per row at a time, persistent over rows):
+//   pass 1  128-bit loads of the row; every thread keeps a running maximum M_t and the sum of
+//           2^((x - M_t) log2 e) over its elements EXCLUDING one instance of its maximum, so that
+//           a row dominated by one logit keeps full relative accuracy in Z - 1 (and hence in
+//           1 - p for the dominating token);
+//   reduce  block maximum, then the block sum rescaled to it, in fp64;
+//   scalar  one thread: logp, rho, clipped surrogate, KL term, the factor g_t of the gradient row
+//           (all fp64), the row's weighted loss term into the workspace;
+//   pass 2  re-read the row (it was just read: served by L2), write bf16(g_t (onehot - softmax)).
+//           Rows whose g_t is exactly 0 (masked, or clipped with no KL term) are written as zeros
+//           without being re-read.
+// Loss reduction: a single CTA sums the chunk's per-row terms in a fixed order (deterministic).
+
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "pods_common.cuh"
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct RowShared {
+    float red_f[32];
+    double red_d[32];
+    int red_i[32];
+    float row_max;
+    double zprime;      // sum over the row of e^(x - max), one instance of the maximum excluded
+    int nmax_threads;
+    float coef;         // -g_t / Z
+    float target;       // g_t (1 - p_token)
+    int write_mode;     // 0: zeros, 1: gradient
+    int token;
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint16_t to_bf16_bits(float v) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Running (max, sum) of one thread: s = sum of 2^(x log2e - mxc) over the thread's elements except
+// one instance of the maximum, where the reference exponent mxc = fl(mx log2e) is an fp32 number in
+// its own right.  The fused multiply-add x*log2e - mxc is then rounded once, and the difference
+// lo = mx*log2e - mxc (exact in fp32, from one more fma) is applied to the finished sum as the
+// factor 2^(-lo), so the rounding of mx*log2e never enters the row's statistics.
+struct OnlineStat {
+    float mx;    // running maximum of the raw logits (-inf before the first element)
+    float mxc;   // fl(mx * log2(e))
+    float s;
+};
+
+// 2^(-lo) for lo = mx*log2e - fl(mx*log2e), |lo| < 2^-18: first-order expansion, fp64.
+__device__ __forceinline__ double ref_correction(float mx, float mxc) {
+    return 1.0 - (double)fmaf(mx, kLog2e, -mxc) * 0.6931471805599453;
+}
+
+__device__ __forceinline__ void stat_add_slow(OnlineStat& st, const float* v, int cnt, float vmax) {
+    // A new maximum arrived: the old maximum becomes an ordinary element (worth 2^lo relative to
+    // the old reference), the sum moves to the new reference, and the first instance of the new
+    // maximum is left out of the sum.
+    const float ref = vmax * kLog2e;
+    if (st.mx != -INFINITY) {
+        const float lo_old = fmaf(st.mx, kLog2e, -st.mxc);
+        st.s = (st.s + fmaf(lo_old, kLn2, 1.0f)) * ex2_approx(st.mxc - ref);
+    }
+    st.mx = vmax;
+    st.mxc = ref;
+    bool skipped = false;
+    for (int i = 0; i < cnt; ++i) {
+        if (!skipped && v[i] == vmax) { skipped = true; continue; }
+        st.s += ex2_approx(fmaf(v[i], kLog2e, -st.mxc));
+    }
+}
+
+__device__ __forceinline__ void stat_add8(OnlineStat& st, const uint4& q) {
+    float v[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                  bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+    const float vmax = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
+    if (vmax > st.mx) {
+        stat_add_slow(st, v, 8, vmax);
+    } else {
+        float a = 0.0f, b = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            a += ex2_approx(fmaf(v[i], kLog2e, -st.mxc));
+            b += ex2_approx(fmaf(v[i + 1], kLog2e, -st.mxc));
+        }
+        st.s += a + b;
+    }
+}
+
+__device__ __forceinline__ void stat_add1(OnlineStat& st, float v) {
+    if (v > st.mx) stat_add_slow(st, &v, 1, v);
+    else st.s += ex2_approx(fmaf(v, kLog2e, -st.mxc));
+}
+
+template <int BLOCK>
+__device__ __forceinline__ float block_max(float v, RowShared& sh) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(PODS_FULL_MASK, v, d));
+    if (lane == 0) sh.red_f[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        float w = lane < BLOCK / 32 ? sh.red_f[lane] : -INFINITY;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) w = fmaxf(w, __shfl_xor_sync(PODS_FULL_MASK, w, d));
+        if (lane == 0) sh.row_max = w;
+    }
+    __syncthreads();
+    return sh.row_max;
+}
+
+template <int BLOCK>
+__device__ __forceinline__ void block_sum(double v, int c, RowShared& sh) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        v += __shfl_xor_sync(PODS_FULL_MASK, v, d);
+        c += __shfl_xor_sync(PODS_FULL_MASK, c, d);
+    }
+    if (lane == 0) { sh.red_d[warp] = v; sh.red_i[warp] = c; }
+    __syncthreads();
+    if (warp == 0) {
+        double w = lane < BLOCK / 32 ? sh.red_d[lane] : 0.0;
+        int k = lane < BLOCK / 32 ? sh.red_i[lane] : 0;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            w += __shfl_xor_sync(PODS_FULL_MASK, w, d);
+            k += __shfl_xor_sync(PODS_FULL_MASK, k, d);
+        }
+        if (lane == 0) { sh.zprime = w; sh.nmax_threads = k; }
+    }
+    __syncthreads();
+}
+
+struct RowArgs {
+    const uint16_t* logits;
+    int64_t ldl;
+    const int32_t* tokens;
+    const float* old_logp;
+    const float* ref_logp;
+    const float* adv;
+    const double* seq_weight;
+    const int64_t* cu_seqlens;
+    int64_t M;
+    int64_t row0;
+    const uint8_t* mask;
+    int64_t T;
+    int32_t V;
+    float eps, beta, grad_scale;
+    float* logp;
+    uint16_t* dlogits;
+    int64_t ldd;
+    double* row_loss;      // workspace [T]: mask_t w_i loss_t
+    uint32_t* status;
+    int vec_ok;            // 16-byte aligned rows: 128-bit path
+};
+
+// Rollout of packed row r: the i with cu_seqlens[i] <= r < cu_seqlens[i+1].
+__device__ __forceinline__ int64_t find_rollout(const int64_t* cu, int64_t M, int64_t r) {
+    int64_t lo = 0, hi = M;            // invariant: cu[lo] <= r, answer in [lo, hi)
+    while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (cu[mid] <= r) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+grpo_loss_rows_kernel(const RowArgs a) {
+    __shared__ RowShared sh;
+    const int tid = threadIdx.x;
+    const int V = a.V;
+    const int nvec = a.vec_ok ? V / 8 : 0;
+
+    for (int64_t t = blockIdx.x; t < a.T; t += gridDim.x) {
+        const uint16_t* row = a.logits + t * a.ldl;
+        uint16_t* drow = a.dlogits + t * a.ldd;
+        const uint4* row4 = reinterpret_cast<const uint4*>(row);
+
+        float x_tok = 0.0f;
+        if (tid == 0) {
+            int tok = a.tokens[t];
+            if (tok < 0 || tok >= V) { tok = 0; pods_raise(a.status, PODS_STATUS_TOKEN_RANGE); }
+            sh.token = tok;
+            x_tok = __uint_as_float((uint32_t)row[tok] << 16);   // read before anything is written in place
+        }
+
+        // ---- pass 1: per-thread running maximum and sum -------------------------------------
+        OnlineStat st = {-INFINITY, -INFINITY, 0.0f};
+        for (int v = tid; v < nvec; v += BLOCK) stat_add8(st, row4[v]);
+        for (int v = nvec * 8 + tid; v < V; v += BLOCK) stat_add1(st, __uint_as_float((uint32_t)row[v] << 16));
+
+        const float mx = block_max<BLOCK>(st.mx, sh);
+        double contrib = 0.0;
+        int is_max = 0;
+        if (st.mx != -INFINITY) {
+            const double s_true = (double)st.s * ref_correction(st.mx, st.mxc);
+            if (st.mx == mx) { contrib = s_true; is_max = 1; }
+            else contrib = (s_true + 1.0) * (double)ex2_approx((st.mx - mx) * kLog2e);
+        }
+        block_sum<BLOCK>(contrib, is_max, sh);
+
+        // ---- scalar terms of the row (one thread, fp64) ---------------------------------------
+        if (tid == 0) {
+            const double zp = sh.zprime + (double)(sh.nmax_threads - 1);   // all but one instance of the max
+            const double Z = 1.0 + zp;
+            const double logp = ((double)x_tok - (double)mx) - log1p(zp);
+            const int64_t i = find_rollout(a.cu_seqlens, a.M, a.row0 + t);
+            const bool live = a.mask == nullptr || a.mask[t] != 0;
+            const double w = live ? a.seq_weight[i] : 0.0;
+            const double adv = (double)a.adv[i];
+            const double eps = (double)a.eps, beta = (double)a.beta;
+            const double rho = exp(logp - (double)a.old_logp[t]);
+            const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
+            const double s1 = rho * adv, s2 = clipped * adv;
+            double loss = -(s1 < s2 ? s1 : s2);
+            double dl = (s1 <= s2) ? -adv * rho : 0.0;
+            if (a.ref_logp != nullptr && beta != 0.0) {
+                const double d = (double)a.ref_logp[t] - logp;
+                const double ed = exp(d);
+                loss += beta * (ed - d - 1.0);
+                dl += beta * (1.0 - ed);
+            }
+            const double g = (w != 0.0) ? (double)a.grad_scale * w * dl : 0.0;
+            const double one_minus_p = (x_tok == mx) ? zp / Z : -expm1(logp);
+            a.logp[t] = (float)logp;
+            a.row_loss[t] = (w != 0.0) ? w * loss : 0.0;    // a masked row adds nothing, whatever its inputs
+            sh.coef = (float)(-g / Z * ref_correction(mx, mx * kLog2e));   // pass 2 uses fl(mx log2e) again
+            sh.target = (float)(g * one_minus_p);
+            sh.write_mode = (g != 0.0) ? 1 : 0;
+        }
+        __syncthreads();
+
+        // ---- pass 2: the gradient row ---------------------------------------------------------
+        const int tok = sh.token;
+        if (sh.write_mode == 0) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            uint4* d4 = reinterpret_cast<uint4*>(drow);
+            for (int v = tid; v < nvec; v += BLOCK) __stcs(d4 + v, z);
+            for (int v = nvec * 8 + tid; v < V; v += BLOCK) drow[v] = 0;
+        } else {
+            const float coef = sh.coef;
+            const float mxc = mx * kLog2e;
+            const uint16_t target_bits = to_bf16_bits(sh.target);
+            uint4* d4 = reinterpret_cast<uint4*>(drow);
+            const int tok_vec = tok >> 3;
+            for (int v = tid; v < nvec; v += BLOCK) {
+                const uint4 q = row4[v];
+                uint4 o;
+                o.x = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.x), kLog2e, -mxc)),
+                                  coef * ex2_approx(fmaf(bf16_hi(q.x), kLog2e, -mxc)));
+                o.y = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.y), kLog2e, -mxc)),
+                                  coef * ex2_approx(fmaf(bf16_hi(q.y), kLog2e, -mxc)));
+                o.z = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.z), kLog2e, -mxc)),
+                                  coef * ex2_approx(fmaf(bf16_hi(q.z), kLog2e, -mxc)));
+                o.w = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.w), kLog2e, -mxc)),
+                                  coef * ex2_approx(fmaf(bf16_hi(q.w), kLog2e, -mxc)));
+                if (v == tok_vec) {
+                    uint32_t* ow = &o.x;
+                    const int e = tok & 7;
+                    const uint32_t shift = (e & 1) ? 16u : 0u;
+                    ow[e >> 1] = (ow[e >> 1] & ~(0xffffu << shift)) | ((uint32_t)target_bits << shift);
+                }
+                __stcs(d4 + v, o);
+            }
+            for (int v = nvec * 8 + tid; v < V; v += BLOCK) {
+                const float x = __uint_as_float((uint32_t)row[v] << 16);
+                drow[v] = (v == tok) ? target_bits : to_bf16_bits(coef * ex2_approx(fmaf(x, kLog2e, -mxc)));
+            }
+        }
+        __syncthreads();     // sh is reused by the next row
+    }
+}
+
+// Fixed-order sum of the chunk's per-row loss terms, added to the accumulator.
+__global__ void __launch_bounds__(1024)
+loss_reduce_kernel(const double* __restrict__ row_loss, int64_t T, double* loss_acc) {
+    __shared__ double part[1024];
+    double s = 0.0;
+    for (int64_t t = threadIdx.x; t < T; t += 1024) s += row_loss[t];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int d = 512; d > 0; d >>= 1) {
+        if ((int)threadIdx.x < d) part[threadIdx.x] += part[threadIdx.x + d];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *loss_acc += part[0];
+}
+
+__global__ void loss_zero_kernel(double* loss_acc) { *loss_acc = 0.0; }
+
+__global__ void loss_finalize_kernel(const double* loss_acc, float* loss) { *loss = (float)*loss_acc; }
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" size_t grpo_loss_chunk_workspace_bytes(int64_t T_chunk) {
+    if (T_chunk < 0) return 0;
+    return align_up((size_t)T_chunk * sizeof(double), 256) + 256;
+}
+
+extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
+                               const float* ref_logp, const float* adv, const double* seq_weight,
+                               const int64_t* cu_seqlens, int64_t M, int64_t row0, const uint8_t* mask,
+                               int64_t T_chunk, int32_t V, float eps, float beta, float grad_scale,
+                               double* loss_acc, float* logp, void* dlogits, int64_t ldd, void* workspace,
+                               size_t workspace_bytes, uint32_t* status, void* stream) {
+    if (T_chunk < 0 || V < 1 || M < 1 || row0 < 0 || ldl < V || ldd < V) return PODS_ERR_INVALID_ARG;
+    if (!(eps >= 0.0f) || !(beta == beta)) return PODS_ERR_INVALID_ARG;
+    if (T_chunk == 0) return PODS_OK;
+    if (logits == nullptr || tokens == nullptr || old_logp == nullptr || adv == nullptr || seq_weight == nullptr ||
+        cu_seqlens == nullptr || loss_acc == nullptr || logp == nullptr || dlogits == nullptr)
+        return PODS_ERR_INVALID_ARG;
+    if (ref_logp == nullptr && beta != 0.0f) return PODS_ERR_INVALID_ARG;
+    if (!pods_aligned(logits, 2) || !pods_aligned(dlogits, 2) || !pods_aligned(loss_acc, 8)) return PODS_ERR_INVALID_ARG;
+    if (dlogits == logits && ldd != ldl) return PODS_ERR_INVALID_ARG;
+    if (workspace == nullptr || workspace_bytes < grpo_loss_chunk_workspace_bytes(T_chunk) ||
+        !pods_aligned(workspace, 16))
+        return PODS_ERR_WORKSPACE;
+
+    RowArgs a;
+    a.logits = static_cast<const uint16_t*>(logits);
+    a.ldl = ldl;
+    a.tokens = tokens;
+    a.old_logp = old_logp;
+    a.ref_logp = ref_logp;
+    a.adv = adv;
+    a.seq_weight = seq_weight;
+    a.cu_seqlens = cu_seqlens;
+    a.M = M;
+    a.row0 = row0;
+    a.mask = mask;
+    a.T = T_chunk;
+    a.V = V;
+    a.eps = eps;
+    a.beta = beta;
+    a.grad_scale = grad_scale;
+    a.logp = logp;
+    a.dlogits = static_cast<uint16_t*>(dlogits);
+    a.ldd = ldd;
+    a.row_loss = static_cast<double*>(workspace);
+    a.status = status;
+    a.vec_ok = pods_aligned(logits, 16) && pods_aligned(dlogits, 16) && ldl % 8 == 0 && ldd % 8 == 0;
+
+    cudaStream_t s = pods_stream(stream);
+    constexpr int BLOCK = 1024;
+    const int64_t cap = (int64_t)pods_sm_count();
+    const int grid = (int)(T_chunk < cap ? T_chunk : cap);
+    grpo_loss_rows_kernel<BLOCK><<<grid, BLOCK, 0, s>>>(a);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    loss_reduce_kernel<<<1, 1024, 0, s>>>(a.row_loss, T_chunk, loss_acc);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
+extern "C" size_t grpo_loss_workspace_bytes(int64_t T, int64_t M, int64_t chunk_rows) {
+    if (T < 0 || M < 0) return 0;
+    const int64_t rows = (chunk_rows <= 0 || chunk_rows > T) ? T : chunk_rows;
+    return grpo_loss_chunk_workspace_bytes(rows) + align_up((size_t)M * sizeof(double), 256) + 256;
+}
+
+extern "C" int grpo_loss_fwd_bwd(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
+                                 const float* ref_logp, const float* adv, const int64_t* cu_seqlens, int64_t M,
+                                 const uint8_t* mask, int64_t T, int32_t V, float eps, float beta,
+                                 int64_t chunk_rows, float* loss, float* logp, void* dlogits, int64_t ldd,
+                                 void* workspace, size_t workspace_bytes, uint32_t* status, void* stream) {
+    if (T < 0 || M < 1 || loss == nullptr) return PODS_ERR_INVALID_ARG;
+    if (workspace == nullptr || workspace_bytes < grpo_loss_workspace_bytes(T, M, chunk_rows) ||
+        !pods_aligned(workspace, 16))
+        return PODS_ERR_WORKSPACE;
+    const int64_t rows = (chunk_rows <= 0 || chunk_rows > T) ? T : chunk_rows;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    double* loss_acc = reinterpret_cast<double*>(ws);
+    double* seq_weight = reinterpret_cast<double*>(ws + 256);
+    unsigned char* chunk_ws = ws + 256 + align_up((size_t)M * sizeof(double), 256);
+    const size_t chunk_ws_bytes = grpo_loss_chunk_workspace_bytes(rows);
+    cudaStream_t s = pods_stream(stream);
+
+    loss_zero_kernel<<<1, 1, 0, s>>>(loss_acc);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    int rc = grpo_seq_weights(mask, cu_seqlens, M, seq_weight, stream);
+    if (rc != PODS_OK) return rc;
+    const uint16_t* lg = static_cast<const uint16_t*>(logits);
+    uint16_t* dl = static_cast<uint16_t*>(dlogits);
+    for (int64_t r0 = 0; r0 < T; r0 += rows) {
+        const int64_t cnt = (T - r0 < rows) ? T - r0 : rows;
+        rc = grpo_loss_chunk(lg + r0 * ldl, ldl, tokens + r0, old_logp + r0, ref_logp ? ref_logp + r0 : nullptr,
+                             adv, seq_weight, cu_seqlens, M, r0, mask ? mask + r0 : nullptr, cnt, V, eps, beta,
+                             1.0f, loss_acc, logp + r0, dl + r0 * ldd, ldd, chunk_ws, chunk_ws_bytes, status,
+                             stream);
+        if (rc != PODS_OK) return rc;
+    }
+    return grpo_loss_finalize(loss_acc, loss, stream);
+}
+
+extern "C" int grpo_loss_finalize(const double* loss_acc, float* loss, void* stream) {
+    if (loss_acc == nullptr || loss == nullptr) return PODS_ERR_INVALID_ARG;
+    loss_finalize_kernel<<<1, 1, 0, pods_stream(stream)>>>(loss_acc, loss);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}

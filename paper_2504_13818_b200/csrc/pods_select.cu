@@ -1,0 +1,347 @@
+// pods_select: the down-sampling rule D(o, r; m) -> S (Definition 3.1) for G prompt groups per
+// launch, and the advantages of the kept subset (Section 3.2).
+//
+// One group is handled by LANES consecutive lanes of a warp (8, 16 or 32), each lane holding E
+// elements in registers (LANES * E >= n, padded with +infinity keys).  Steps, per group:
+//   1. load the rewards (coalesced), build a 64-bit key (order-preserving reward bits : index)
+//      so that one unsigned compare gives the stable (reward, index) order of argsort;
+//   2. bitonic sort: strides below E are compare-exchanges between registers of a lane, larger
+//      strides exchange with another lane by shuffle (Algorithm 2, step 1);
+//   3. fp64 running sums of the centred rewards and their squares over the sorted order, upward
+//      from the lowest and downward from the highest, written to shared memory (the prefix sums
+//      of Theorem 1's proof);
+//   4. each lane scores its share of the m+1 splits "k highest + (m-k) lowest" from the prefix
+//      sums, then a shuffle arg-max picks the largest score, smallest k (Algorithm 2, steps 2-6);
+//   5. kept elements are marked in a bitmap indexed by original index, then written out in
+//      ascending original index with a ballot compaction, together with their advantages.
+
+#include <math.h>
+
+#include "pods_common.cuh"
+
+namespace {
+
+constexpr int kSelectWarps = 4;                 // warps per CTA
+constexpr int kSelectThreads = kSelectWarps * 32;
+
+// Philox4x32-10 (Salmon et al., SC'11): 10 rounds of two 32x32->64 multiplies and key bumps.
+__device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                      uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ k0;
+        const uint32_t n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+// fp32 -> uint32 whose unsigned order is the order of the floats; -0 is folded into +0 and every
+// NaN becomes the largest key below the padding sentinel.
+__device__ __forceinline__ uint32_t ordered_bits(float r) {
+    uint32_t u = __float_as_uint(r);
+    if ((u << 1) == 0u) u = 0u;                              // -0 -> +0
+    if ((u & 0x7fffffffu) > 0x7f800000u) u = 0x7fffffffu;    // any NaN -> one positive NaN
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float from_ordered_bits(uint32_t o) {
+    const uint32_t u = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+    return __uint_as_float(u);
+}
+
+// Shared memory of one group: prefix sums at sorted positions 0..m and suffix sums at positions
+// n-m..n of the centred rewards and their squares (fp64), a copy of the rewards (random rule only),
+// and two bitmaps (kept original indices, kept sorted positions).
+struct SelectSmemLayout {
+    int slot_bytes;
+    int rbuf_off, sel_off, pos_off;
+};
+
+__host__ __device__ inline SelectSmemLayout select_layout(int npad, int m) {
+    SelectSmemLayout L;
+    const int words = npad >= 32 ? npad / 32 : 1;
+    L.rbuf_off = 4 * (m + 1) * 8;
+    L.sel_off = L.rbuf_off + npad * 4;
+    L.pos_off = L.sel_off + words * 4;
+    L.slot_bytes = (L.pos_off + words * 4 + 7) & ~7;
+    return L;
+}
+
+template <int LANES, int E>
+__global__ void __launch_bounds__(kSelectThreads)
+pods_select_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint64_t seed,
+                   uint32_t flags, int32_t* __restrict__ idx_out, float* __restrict__ adv_out,
+                   int32_t* __restrict__ k_out, uint32_t* status) {
+    constexpr int NPAD = LANES * E;
+    constexpr int GPW = 32 / LANES;                 // groups per warp
+    constexpr int WORDS = NPAD >= 32 ? NPAD / 32 : 1;
+    constexpr uint32_t GROUP_MASK = LANES == 32 ? 0xffffffffu : ((1u << LANES) - 1u);
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / LANES, sl = lane % LANES;
+    const SelectSmemLayout lay = select_layout(NPAD, m);
+    unsigned char* slot = smem_raw + (size_t)(warp * GPW + sub) * lay.slot_bytes;
+    double* PL1 = reinterpret_cast<double*>(slot);      // sum of the j lowest,  j = 0..m
+    double* PL2 = PL1 + (m + 1);
+    double* SU1 = PL2 + (m + 1);                        // sum of the m-j highest, j = 0..m
+    double* SU2 = SU1 + (m + 1);
+    float* rbuf = reinterpret_cast<float*>(slot + lay.rbuf_off);
+    uint32_t* sel = reinterpret_cast<uint32_t*>(slot + lay.sel_off);
+    uint32_t* possel = reinterpret_cast<uint32_t*>(slot + lay.pos_off);
+
+    const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
+    for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
+        const int64_t g = base + sub;
+        const bool valid = g < G;
+        const float* r_g = rewards + (valid ? g : 0) * (int64_t)n;
+
+        // ---- 1. load and key ------------------------------------------------------------------
+        uint64_t key[E];
+        bool nonfinite = false;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int i = e * LANES + sl;                    // original index (coalesced load)
+            key[e] = 0xffffffffffffffffull;                  // padding sorts last
+            if (i < n) {
+                const float r = valid ? r_g[i] : 0.0f;
+                nonfinite |= !(fabsf(r) <= 3.402823466e38f);
+                uint32_t hi;
+                if (rule == PODS_RULE_RANDOM) {
+                    rbuf[i] = r;
+                    hi = philox_first_word((uint32_t)i, 0u, (uint32_t)((uint64_t)g & 0xffffffffu),
+                                           (uint32_t)((uint64_t)g >> 32), (uint32_t)(seed & 0xffffffffu),
+                                           (uint32_t)(seed >> 32));
+                } else {
+                    hi = ordered_bits(r);
+                }
+                key[e] = ((uint64_t)hi << 32) | (uint32_t)i;
+            }
+        }
+        if (nonfinite && valid) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
+
+        // ---- 2. bitonic sort over positions p = sl * E + e ------------------------------------
+#pragma unroll
+        for (int k = 2; k <= NPAD; k <<= 1) {
+#pragma unroll
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                if (j >= E) {
+                    const int lane_xor = j / E;
+                    const bool lower = (sl & lane_xor) == 0;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const bool up = ((sl * E + e) & k) == 0;
+                        const uint64_t other = __shfl_xor_sync(PODS_FULL_MASK, key[e], lane_xor);
+                        const uint64_t lo = key[e] < other ? key[e] : other;
+                        const uint64_t hi = key[e] < other ? other : key[e];
+                        key[e] = (lower == up) ? lo : hi;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if ((e & j) == 0) {
+                            const bool up = ((sl * E + e) & k) == 0;
+                            const uint64_t a = key[e], b = key[e | j];
+                            const uint64_t lo = a < b ? a : b;
+                            const uint64_t hi = a < b ? b : a;
+                            key[e] = up ? lo : hi;
+                            key[e | j] = up ? hi : lo;
+                        }
+                    }
+                }
+            }
+        }
+
+        // ---- 3. centred rewards and fp64 prefix sums over the sorted order ------------------
+        double x[E];
+        double centre;
+        if (rule == PODS_RULE_RANDOM) {
+            __syncwarp();
+            centre = (double)rbuf[0];
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int p = sl * E + e;
+                x[e] = p < n ? (double)rbuf[(uint32_t)key[e]] - centre : 0.0;
+            }
+        } else {
+            const uint64_t first = __shfl_sync(PODS_FULL_MASK, key[0], sub * LANES);
+            centre = (double)from_ordered_bits((uint32_t)(first >> 32));     // the group minimum
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int p = sl * E + e;
+                x[e] = p < n ? (double)from_ordered_bits((uint32_t)(key[e] >> 32)) - centre : 0.0;
+            }
+        }
+
+        int kstar = -1;
+        if (rule == PODS_RULE_MAXVAR && m < n) {
+            double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) { s1 += x[e]; s2 += x[e] * x[e]; }
+            double i1 = s1, i2 = s2;                         // inclusive scan over the lanes below
+            double j1 = s1, j2 = s2;                         // inclusive scan over the lanes above
+#pragma unroll
+            for (int d = 1; d < LANES; d <<= 1) {
+                const double t1 = __shfl_up_sync(PODS_FULL_MASK, i1, d, LANES);
+                const double t2 = __shfl_up_sync(PODS_FULL_MASK, i2, d, LANES);
+                const double u1 = __shfl_down_sync(PODS_FULL_MASK, j1, d, LANES);
+                const double u2 = __shfl_down_sync(PODS_FULL_MASK, j2, d, LANES);
+                if (sl >= d) { i1 += t1; i2 += t2; }
+                if (sl + d < LANES) { j1 += u1; j2 += u2; }
+            }
+            // Both ends are summed directly (lowest upward, highest downward): no split score is a
+            // difference of running totals, so equal splits score equal and nothing cancels.
+            double a1 = i1 - s1, a2 = i2 - s2;               // sum over positions below this lane's first
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int p = sl * E + e;
+                if (p <= m) { PL1[p] = a1; PL2[p] = a2; }
+                a1 += x[e];
+                a2 += x[e] * x[e];
+            }
+            double b1 = j1 - s1, b2 = j2 - s2;               // sum over positions above this lane's last
+            if (sl == LANES - 1 && n == NPAD) { SU1[m] = 0.0; SU2[m] = 0.0; }
+#pragma unroll
+            for (int e = E - 1; e >= 0; --e) {
+                const int p = sl * E + e;
+                b1 += x[e];
+                b2 += x[e] * x[e];
+                if (p >= n - m && p <= n) { SU1[p - (n - m)] = b1; SU2[p - (n - m)] = b2; }
+            }
+            __syncwarp();
+
+            // ---- 4. score the splits: m^2 Var = m * sum x^2 - (sum x)^2 ----------------------
+            double best = -INFINITY;
+            int bestk = 0x7fffffff;
+            for (int k = sl; k <= m; k += LANES) {
+                const double q1 = PL1[m - k] + SU1[m - k];
+                const double q2 = PL2[m - k] + SU2[m - k];
+                // separately rounded products (no fused multiply-add): equal sums give equal scores
+                const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
+                if (score > best || bestk == 0x7fffffff) { best = score; bestk = k; }
+            }
+#pragma unroll
+            for (int d = LANES >> 1; d > 0; d >>= 1) {
+                const double ob = __shfl_xor_sync(PODS_FULL_MASK, best, d);
+                const int ok = __shfl_xor_sync(PODS_FULL_MASK, bestk, d);
+                if (ok != 0x7fffffff && (bestk == 0x7fffffff || ob > best || (ob == best && ok < bestk))) {
+                    best = ob;
+                    bestk = ok;
+                }
+            }
+            kstar = __shfl_sync(PODS_FULL_MASK, bestk, sub * LANES);   // one verdict per group, even with NaN scores
+            __syncwarp();
+        } else if (rule == PODS_RULE_MAXVAR) {
+            kstar = 0;                                       // m == n: every split is the whole group
+        } else if (rule == PODS_RULE_MAXREWARD) {
+            kstar = m;
+        }
+
+        // ---- 5. mark the kept elements ----------------------------------------------------------
+        for (int w = sl; w < WORDS; w += LANES) { sel[w] = 0u; possel[w] = 0u; }
+        __syncwarp();
+        if (rule == PODS_RULE_PERCENTILE) {
+            for (int j = sl; j < m; j += LANES) {
+                const int pos = (int)(((2 * (int64_t)j + 1) * n) / (2 * (int64_t)m));
+                atomicOr(&possel[pos >> 5], 1u << (pos & 31));
+            }
+            __syncwarp();
+        }
+        double s1 = 0.0, s2 = 0.0, f1 = 0.0, f2 = 0.0;      // sums over the kept subset / the full group
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int p = sl * E + e;
+            bool keep;
+            if (rule == PODS_RULE_PERCENTILE) keep = p < n && ((possel[p >> 5] >> (p & 31)) & 1u);
+            else if (rule == PODS_RULE_RANDOM) keep = p < m;
+            else keep = p < m - kstar || (p >= n - kstar && p < n);
+            if (keep) {
+                const uint32_t i = (uint32_t)key[e];
+                atomicOr(&sel[i >> 5], 1u << (i & 31));
+                s1 += x[e];
+                s2 += x[e] * x[e];
+            }
+            f1 += x[e];
+            f2 += x[e] * x[e];
+        }
+        if (flags & PODS_FLAG_ADV_BEFORE) { s1 = f1; s2 = f2; }
+#pragma unroll
+        for (int d = LANES >> 1; d > 0; d >>= 1) {
+            s1 += __shfl_xor_sync(PODS_FULL_MASK, s1, d);
+            s2 += __shfl_xor_sync(PODS_FULL_MASK, s2, d);
+        }
+        __syncwarp();
+
+        // advantages: a = (x - S/c) / sigma with sigma^2 = (c Q - S^2) / (c d), d = c or c - 1
+        const double cnt = (flags & PODS_FLAG_ADV_BEFORE) ? (double)n : (double)m;
+        const double den = (flags & PODS_FLAG_STD_SAMPLE) ? cnt - 1.0 : cnt;
+        const double J = __dsub_rn(__dmul_rn(cnt, s2), __dmul_rn(s1, s1));
+        const double inv_sigma_c = (J > 0.0 && den > 0.0) ? sqrt(den / (cnt * J)) : 0.0;   // 1 / (c sigma)
+
+        // ---- 6. emit in ascending original index ------------------------------------------------
+        int written = 0;
+        for (int i0 = 0; i0 < n; i0 += LANES) {
+            const int i = i0 + sl;
+            const bool bit = i < n && ((sel[i >> 5] >> (i & 31)) & 1u);
+            const uint32_t ballot = __ballot_sync(PODS_FULL_MASK, bit);
+            const uint32_t mine = (ballot >> (sub * LANES)) & GROUP_MASK;
+            if (bit && valid) {
+                const int off = written + __popc(mine & ((1u << sl) - 1u));
+                const double xi = (double)r_g[i] - centre;
+                idx_out[g * (int64_t)m + off] = i;
+                adv_out[g * (int64_t)m + off] = (float)((xi * cnt - s1) * inv_sigma_c);
+            }
+            written += __popc(mine);
+        }
+        if (valid && sl == 0 && k_out != nullptr) k_out[g] = kstar;
+        __syncwarp();
+    }
+}
+
+template <int LANES, int E>
+int launch_select(const float* rewards, int64_t G, int n, int m, int rule, uint64_t seed, uint32_t flags,
+                  int32_t* idx, float* adv, int32_t* k_out, uint32_t* status, cudaStream_t stream) {
+    constexpr int GPW = 32 / LANES;
+    const SelectSmemLayout lay = select_layout(LANES * E, m);
+    const size_t smem = (size_t)lay.slot_bytes * kSelectWarps * GPW;
+    auto kernel = pods_select_kernel<LANES, E>;
+    if (smem > 48 * 1024)
+        PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t groups_per_cta = (int64_t)kSelectWarps * GPW;
+    const int64_t needed = (G + groups_per_cta - 1) / groups_per_cta;
+    const int64_t cap = (int64_t)pods_sm_count() * 16;
+    const int grid = (int)(needed < cap ? needed : cap);
+    kernel<<<grid, kSelectThreads, smem, stream>>>(rewards, G, n, m, rule, seed, flags, idx, adv, k_out, status);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
+}  // namespace
+
+extern "C" int pods_select(const float* rewards, int64_t G, int32_t n, int32_t m, int32_t rule, uint64_t seed,
+                           uint32_t flags, int32_t* idx, float* adv, int32_t* k_out, uint32_t* status,
+                           void* stream) {
+    if (G < 0 || n < 1 || m < 1 || m > n) return PODS_ERR_INVALID_ARG;
+    if (rule < PODS_RULE_MAXVAR || rule > PODS_RULE_PERCENTILE) return PODS_ERR_UNSUPPORTED;
+    if (n > PODS_MAX_N) return PODS_ERR_UNSUPPORTED;
+    if (G == 0) return PODS_OK;
+    if (rewards == nullptr || idx == nullptr || adv == nullptr) return PODS_ERR_INVALID_ARG;
+    if (!pods_aligned(rewards, 4) || !pods_aligned(idx, 4) || !pods_aligned(adv, 4)) return PODS_ERR_INVALID_ARG;
+    cudaStream_t s = pods_stream(stream);
+#define PODS_SELECT_CASE(LANES, E) \
+    return launch_select<LANES, E>(rewards, G, n, m, rule, seed, flags, idx, adv, k_out, status, s)
+    if (n <= 8) PODS_SELECT_CASE(8, 1);
+    if (n <= 16) PODS_SELECT_CASE(16, 1);
+    if (n <= 32) PODS_SELECT_CASE(32, 1);
+    if (n <= 64) PODS_SELECT_CASE(32, 2);
+    if (n <= 128) PODS_SELECT_CASE(32, 4);
+    if (n <= 256) PODS_SELECT_CASE(32, 8);
+    if (n <= 512) PODS_SELECT_CASE(32, 16);
+    PODS_SELECT_CASE(32, 32);
+#undef PODS_SELECT_CASE
+}

@@ -1,0 +1,185 @@
+"""grpo_loss_fwd_bwd / grpo_loss_chunk (CUDA) against the oracle.
+
+Bar: per-token log-prob abs <= 1e-3, loss rel <= 1e-4 (see parity.assert_loss_close for sums that
+cancel), dlogits within 2 bf16 ulps.  Rows whose
+min(rho a, clip(rho) a) is within CLIP_MARGIN of switching branch are compared on logp only (the
+branch is a floating-point decision; none is expected with these inputs and the count is asserted)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_13818_b200 import binding, workloads as wl
+from parity import (CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, assert_loss_close, build_batch, dlogits_ulp_error,
+                    gradient_slack, oracle_loss, shrink)
+
+pytestmark = pytest.mark.gpu
+
+
+def _t(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    return (t if dtype is None else t.view(dtype)).cuda()
+
+
+def _gpu_loss(b, chunk_rows=0, in_place=False, ref=True, beta=None, mask=None):
+    w = b["w"]
+    logits = _t(b["logits"], torch.bfloat16)
+    status = binding.new_status()
+    dlogits = logits if in_place else None
+    loss, logp, dl = binding.grpo_loss_fwd_bwd(
+        logits, _t(b["tokens"]), _t(b["old"]), _t(b["ref"]) if ref else None, _t(b["adv32"]),
+        _t(b["mask"] if mask is None else mask) if mask is not False else None,
+        w.eps, w.beta if beta is None else beta, _t(b["cu"]), chunk_rows=chunk_rows, dlogits=dlogits, status=status)
+    torch.cuda.synchronize()
+    return (float(loss.item()), logp.cpu().numpy(), dl.view(torch.uint16).cpu().numpy(),
+            binding.read_status(status))
+
+
+def _check(b, got, want, expect_fragile=0):
+    loss, logp, dl_bits, status = got
+    assert status == 0
+    assert np.abs(logp - want["logp"]).max() <= LOGP_ATOL
+    assert_loss_close(loss, want, b)
+    fragile = (want["margin"] < CLIP_MARGIN) & (want["margin"] > 0)
+    assert int(fragile.sum()) == expect_fragile
+    ulps = dlogits_ulp_error(dl_bits, want["dlogits"], gradient_slack(b, want))
+    worst = ulps[~fragile].max() if (~fragile).any() else 0.0
+    assert worst <= DLOGITS_ULPS, "dlogits off by %.2f bf16 ulps" % worst
+    return worst
+
+
+def test_config1_whole_path_values():
+    b = build_batch(wl.WORKLOADS["c1_tiny"])
+    _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 1000, 1024, 8200, 40001])
+def test_vocab_sizes_span_tiles_and_ragged_tails(V):
+    w = shrink(wl.WORKLOADS["c1_tiny"], V=V, G=3, n=8, m=4, seed=V, spike=6.0, spike_frac=0.3)
+    b = build_batch(w)
+    _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+def test_many_rows_more_than_one_wave_and_in_place():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=6, n=8, m=4, V=2048, len_lo=20, len_hi=40, seed=9)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    assert b["tokens"].shape[0] > 2 * 148
+    a = _gpu_loss(b)
+    _check(b, a, want)
+    c = _gpu_loss(b, in_place=True)
+    assert c[2].tobytes() == a[2].tobytes() and c[0] == a[0]
+
+
+def test_chunked_equals_whole_bitwise_on_rows_and_within_tolerance_on_loss():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=5, n=8, m=4, V=512, seed=21)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    whole = _gpu_loss(b)
+    for rows in (1, 7, 64, 100000):
+        part = _gpu_loss(b, chunk_rows=rows)
+        assert part[1].tobytes() == whole[1].tobytes() and part[2].tobytes() == whole[2].tobytes()
+        assert_loss_close(part[0], want, b)
+
+
+def test_masked_rows_and_empty_rollouts():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=3, n=8, m=4, V=264, seed=5)
+    b = build_batch(w)
+    rng = np.random.default_rng(0)
+    b["mask"] = (rng.uniform(size=b["tokens"].shape[0]) < 0.7).astype(np.uint8)
+    b["mask"][b["cu"][2]:b["cu"][3]] = 0                   # one rollout fully masked
+    b["old"][b["mask"] == 0] = np.float32(-1e30)           # garbage under the mask must not leak into the loss
+    want = oracle_loss(b)
+    got = _gpu_loss(b)
+    _check(b, got, want)
+    assert (got[2][b["mask"] == 0] == 0).all()
+
+
+def test_no_reference_policy_when_beta_is_zero():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=3, n=8, m=4, V=520, beta=0.0, seed=6)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    _check(b, _gpu_loss(b, ref=False, mask=False), want)
+    _check(b, _gpu_loss(b), want)
+
+
+def test_clipped_rows_have_exactly_zero_gradient_rows():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=3, n=8, m=4, V=520, beta=0.0, seed=8)
+    b = build_batch(w)
+    a_row = b["adv32"][b["seq_of_row"]]
+    b["old"] = (b["old"] - np.sign(a_row) * 0.5).astype(np.float32)     # rho far on the penalised side
+    want = oracle_loss(b)
+    got = _gpu_loss(b)
+    _check(b, got, want)
+    assert (got[2][a_row != 0] & 0x7fff == 0).all()
+
+
+def test_peaked_rows_keep_relative_accuracy_of_one_minus_p():
+    """A policy that is nearly certain: the target's gradient g (1 - p) is tiny and must still be
+    accurate to 2 bf16 ulps (the sum excludes the maximum, so Z - 1 is not lost to rounding)."""
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=2, n=8, m=4, V=4096, seed=12, logit_sigma=1.0)
+    b = build_batch(w)
+    x = wl.bf16_bits_to_f32(b["logits"])
+    T = x.shape[0]
+    boost = np.linspace(6.0, 24.0, T).astype(np.float32)    # 1 - p down to ~1e-7: fp64 still resolves it
+    x[np.arange(T), b["tokens"]] += boost
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    lt = wl.host_logp_tilde(b["logits"], b["tokens"])
+    b["old"], b["ref"] = wl.make_old_ref(w, lt)
+    want = oracle_loss(b)
+    assert (want["logp"] > -1e-3).sum() > T // 3
+    _check(b, _gpu_loss(b), want)
+
+
+def test_token_out_of_range_sets_status_and_uses_token_zero():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=2, n=8, m=4, V=128, seed=13)
+    b = build_batch(w)
+    b["tokens"] = b["tokens"].copy()
+    b["tokens"][3] = w.V
+    b["tokens"][5] = -1
+    got = _gpu_loss(b)
+    assert got[3] & binding.STATUS_TOKEN_RANGE
+    want = oracle_loss(b)
+    assert want["bad_tokens"] == 2
+    assert np.abs(got[1] - want["logp"]).max() <= LOGP_ATOL
+    assert dlogits_ulp_error(got[2], want["dlogits"], gradient_slack(b, want)).max() <= DLOGITS_ULPS
+
+
+def test_strided_and_misaligned_rows_take_the_elementwise_path():
+    w = shrink(wl.WORKLOADS["c1_tiny"], G=2, n=8, m=4, V=250, seed=14)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    T, V = b["logits"].shape
+    wide = torch.zeros((T, V + 3), dtype=torch.bfloat16, device="cuda")
+    wide[:, 1:V + 1] = _t(b["logits"], torch.bfloat16)
+    view = wide[:, 1:V + 1]                                   # pitch V+3, base off by 2 bytes
+    status = binding.new_status()
+    loss, logp, dl = binding.grpo_loss_fwd_bwd(view, _t(b["tokens"]), _t(b["old"]), _t(b["ref"]), _t(b["adv32"]),
+                                               None, w.eps, w.beta, _t(b["cu"]), status=status)
+    torch.cuda.synchronize()
+    _check(b, (float(loss.item()), logp.cpu().numpy(), dl.view(torch.uint16).cpu().numpy(), 0), want)
+
+
+def test_whole_path_chained_on_its_own_outputs():
+    """select -> compact -> loss on the GPU's own intermediate results equals the oracle's chain."""
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=3000, len_lo=8, len_hi=40)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    idx, adv, _ = binding.pods_select(_t(b["rewards"]), w.m)
+    src_old = np.zeros(b["src_tokens"].shape, np.float32)
+    src_ref = np.zeros(b["src_tokens"].shape, np.float32)
+    for i in range(b["cu"].shape[0] - 1):                     # scatter the packed old/ref back to rollout storage
+        g, j = divmod(i, w.m)
+        row = g * w.n + int(b["sel"]["idx"][g, j])
+        L = int(b["cu"][i + 1] - b["cu"][i])
+        src_old[row, :L] = b["old"][b["cu"][i]:b["cu"][i + 1]]
+        src_ref[row, :L] = b["ref"][b["cu"][i]:b["cu"][i + 1]]
+    cu, toks, (old, ref) = binding.pods_compact(idx, w.n, _t(b["lengths"]), _t(b["src_tokens"]),
+                                                [_t(src_old), _t(src_ref)])
+    T = int(cu[-1].item())
+    assert T == b["tokens"].shape[0]
+    loss, logp, dl = binding.grpo_loss_fwd_bwd(_t(b["logits"], torch.bfloat16), toks[:T].contiguous(),
+                                               old[:T].contiguous(), ref[:T].contiguous(), adv, None,
+                                               w.eps, w.beta, cu, chunk_rows=500)
+    torch.cuda.synchronize()
+    _check(b, (float(loss.item()), logp.cpu().numpy(), dl.view(torch.uint16).cpu().numpy(), 0), want)
