@@ -34,7 +34,8 @@ typedef enum {
     PODS_ERR_INVALID_ARG = 1,   /* bad size, null pointer, misaligned pointer */
     PODS_ERR_UNSUPPORTED = 2,   /* n above PODS_MAX_N, unknown rule */
     PODS_ERR_WORKSPACE = 3,     /* workspace missing or too small */
-    PODS_ERR_CUDA = 4           /* a CUDA runtime call failed (launch, copy) */
+    PODS_ERR_CUDA = 4,          /* a CUDA runtime call failed (launch, copy) */
+    PODS_ERR_STATIC_CAPACITY = 5 /* grpo_loss_chunk_static: more rows than the built-in scratch holds */
 } pods_status;
 
 /* Bits of the device status word. */
@@ -155,6 +156,36 @@ int grpo_loss_fwd_bwd(const void* logits, int64_t ldl, const int32_t* tokens, co
                       const uint8_t* mask, int64_t T, int32_t V, float eps, float beta, int64_t chunk_rows,
                       float* loss, float* logp, void* dlogits, int64_t ldd, void* workspace,
                       size_t workspace_bytes, uint32_t* status, void* stream);
+
+/*
+ * grpo_loss_chunk_static - grpo_loss_chunk without a workspace argument, for callers that must not
+ * allocate device memory and have none to spare: code running inside a framework's memory-planned
+ * region or a plug-in that is handed only its inputs and outputs, an embedder that forbids cudaMalloc
+ * after start-up, a process whose allocator is frozen while a profiler or checkpointer is attached.
+ * (The paper has no counterpart; this is a packaging variant of the same computation.)
+ *
+ * The per-row loss terms that grpo_loss_chunk keeps in the caller's workspace are kept here in a
+ * fixed array inside the library image: grpo_loss_chunk_static_max_rows() rows (16384) of fp64,
+ * 128.5 KB, resident on every GPU that loads the library until the process exits.  The call itself
+ * calls no cudaMalloc, cudaFree or allocating library routine.  Same arguments, outputs and status
+ * bits as grpo_loss_chunk, minus workspace/workspace_bytes.
+ *
+ *   - T_chunk above grpo_loss_chunk_static_max_rows() returns PODS_ERR_STATIC_CAPACITY and launches
+ *     nothing: split the rows into more chunks.
+ *   - The first call on each device looks up the array's device address (a host-side runtime query,
+ *     with that device current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the last call's contents.  Nothing in it
+ *     needs clearing: each call overwrites the T_chunk slots it later sums.  Two calls that can run
+ *     at the same time on the GPU (different streams, no ordering between them) race on it and give
+ *     a wrong loss_acc; order them, or use grpo_loss_chunk with separate workspaces.
+ */
+int64_t grpo_loss_chunk_static_max_rows(void);
+int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
+                           const float* ref_logp, const float* adv, const double* seq_weight,
+                           const int64_t* cu_seqlens, int64_t M, int64_t row0, const uint8_t* mask,
+                           int64_t T_chunk, int32_t V, float eps, float beta, float grad_scale,
+                           double* loss_acc, float* logp, void* dlogits, int64_t ldd, uint32_t* status,
+                           void* stream);
 
 /* Convert the fp64 accumulator of grpo_loss_chunk calls to the fp32 loss.  Both [dev]. */
 int grpo_loss_finalize(const double* loss_acc, float* loss, void* stream);

@@ -32,6 +32,9 @@ SIGNATURES = {
     "grpo_loss_chunk_workspace_bytes": (_sz, [_i64]),
     "grpo_loss_chunk": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _p, _i64, _i64, _p, _i64, _i32, _f32, _f32,
                                   _f32, _p, _p, _p, _i64, _p, _sz, _p, _p]),
+    "grpo_loss_chunk_static_max_rows": (_i64, []),
+    "grpo_loss_chunk_static": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _p, _i64, _i64, _p, _i64, _i32, _f32, _f32,
+                                         _f32, _p, _p, _p, _i64, _p, _p]),
     "grpo_loss_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "grpo_loss_fwd_bwd": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i32, _f32, _f32, _i64,
                                     _p, _p, _p, _i64, _p, _sz, _p, _p]),
@@ -199,6 +202,31 @@ def grpo_loss_chunk(logits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seql
                                 _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
                                 _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_loss_chunk")
+
+
+def grpo_loss_chunk_static_max_rows() -> int:
+    return int(load().grpo_loss_chunk_static_max_rows())
+
+
+def grpo_loss_chunk_static(logits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, row0, mask, eps, beta,
+                           loss_acc, logp, dlogits, grad_scale=1.0, status=None):
+    """grpo_loss_chunk for callers that may not allocate: no workspace, the scratch is inside the library.
+
+    At most grpo_loss_chunk_static_max_rows() rows per call; calls on one device share the scratch, so
+    they must not overlap on the GPU.  This wrapper itself creates no tensor."""
+    lp, ldl = _rows(logits, "logits")
+    dp, ldd = _rows(dlogits, "dlogits")
+    T, V = logits.shape
+    rc = load().grpo_loss_chunk_static(lp, ldl, _dev(tokens, torch.int32, "tokens"),
+                                       _dev(old_logp, torch.float32, "old_logp"),
+                                       _dev(ref_logp, torch.float32, "ref_logp", True),
+                                       _dev(adv.reshape(-1), torch.float32, "adv"),
+                                       _dev(seq_weight, torch.float64, "seq_weight"),
+                                       _dev(cu_seqlens, torch.int64, "cu_seqlens"), cu_seqlens.shape[0] - 1, row0,
+                                       _dev(mask, torch.uint8, "mask", True), T, V, eps, beta, grad_scale,
+                                       _dev(loss_acc, torch.float64, "loss_acc"), _dev(logp, torch.float32, "logp"),
+                                       dp, ldd, _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "grpo_loss_chunk_static")
 
 
 def grpo_loss_finalize(loss_acc, loss):

@@ -423,3 +423,55 @@ extern "C" int grpo_loss_finalize(const double* loss_acc, float* loss, void* str
     PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
     return PODS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// grpo_loss_chunk_static: grpo_loss_chunk for callers that cannot hand over a workspace.
+// ---------------------------------------------------------------------------------------------
+// The per-row loss terms live in a fixed device array that is part of the library image, so the
+// call needs no workspace argument and allocates nothing.
+
+#define PODS_STATIC_CHUNK_ROWS 16384
+
+namespace {
+
+// One fp64 slot per row of the largest chunk, plus the pad the workspace size formula asks for.
+constexpr size_t kStaticScratchBytes = (size_t)PODS_STATIC_CHUNK_ROWS * sizeof(double) + 512;
+static __device__ __align__(256) unsigned char g_static_row_loss[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};     // device address of the array, per device ordinal
+
+// The array's name is only a handle on the host; its device address has to be asked for, on the
+// device that is current.  Done on the first call per device and remembered.
+int static_scratch_address(void** out) {
+    int dev = 0;
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return PODS_ERR_UNSUPPORTED;
+    void* p = __atomic_load_n(&g_static_scratch_ptr[dev], __ATOMIC_ACQUIRE);
+    if (p == nullptr) {
+        PODS_RETURN_IF_CUDA_ERROR(cudaGetSymbolAddress(&p, g_static_row_loss));
+        if (p == nullptr) return PODS_ERR_CUDA;
+        __atomic_store_n(&g_static_scratch_ptr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return PODS_OK;
+}
+
+}  // namespace
+
+extern "C" int64_t grpo_loss_chunk_static_max_rows(void) { return PODS_STATIC_CHUNK_ROWS; }
+
+extern "C" int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* tokens,
+                                      const float* old_logp, const float* ref_logp, const float* adv,
+                                      const double* seq_weight, const int64_t* cu_seqlens, int64_t M,
+                                      int64_t row0, const uint8_t* mask, int64_t T_chunk, int32_t V, float eps,
+                                      float beta, float grad_scale, double* loss_acc, float* logp,
+                                      void* dlogits, int64_t ldd, uint32_t* status, void* stream) {
+    if (T_chunk > PODS_STATIC_CHUNK_ROWS) return PODS_ERR_STATIC_CAPACITY;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != PODS_OK) return rc;
+    return grpo_loss_chunk(logits, ldl, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, M, row0, mask,
+                           T_chunk, V, eps, beta, grad_scale, loss_acc, logp, dlogits, ldd, scratch,
+                           kStaticScratchBytes, status, stream);
+}

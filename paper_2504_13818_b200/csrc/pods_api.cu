@@ -11,6 +11,7 @@ extern "C" const char* pods_status_string(int status) {
         case PODS_ERR_UNSUPPORTED: return "unsupported size or rule";
         case PODS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case PODS_ERR_CUDA: return "CUDA runtime error";
+        case PODS_ERR_STATIC_CAPACITY: return "chunk has more rows than the built-in scratch array holds";
         default: return "unknown status";
     }
 }
