@@ -1,18 +1,19 @@
 // grpo_loss: the GRPO-PODS token objective L_PODS(theta, S) of Section 3.2 and its gradient with
-// respect to the bf16 logits, fused: per row one streaming pass for the softmax statistics and the
-// target log-prob, the scalar loss terms, then the gradient row.
+// respect to the bf16 logits, fused: per row the softmax statistics and the target log-prob, the
+// scalar loss terms, then the gradient row.
 //
-// Row kernel (one CTA per row at a time, persistent over rows):
-//   pass 1  128-bit loads of the row; every thread keeps a running maximum M_t and the sum of
-//           2^((x - M_t) log2 e) over its elements EXCLUDING one instance of its maximum, so that
-//           a row dominated by one logit keeps full relative accuracy in Z - 1 (and hence in
-//           1 - p for the dominating token);
-//   reduce  block maximum, then the block sum rescaled to it, in fp64;
-//   scalar  one thread: logp, rho, clipped surrogate, KL term, the factor g_t of the gradient row
-//           (all fp64), the row's weighted loss term into the workspace;
-//   pass 2  re-read the row (it was just read: served by L2), write bf16(g_t (onehot - softmax)).
-//           Rows whose g_t is exactly 0 (masked, or clipped with no KL term) are written as zeros
-//           without being re-read.
+// Row kernel (one CTA per row at a time, persistent over rows), three uniform sweeps of the row:
+//   max   128-bit loads from HBM, packed bf16x2 maxima; each thread remembers where its maximum
+//         was; a block arg-max gives the row maximum M and the position of its first instance;
+//   sum   the row again (just read: served by L2): sum of 2^(x log2e - ref), ref = fl(M log2e),
+//         over every element EXCEPT that one instance of the maximum, so that a row dominated by
+//         one logit keeps full relative accuracy in Z - 1 (hence in 1 - p of the dominating token);
+//         the exact residual M log2e - ref is applied to the finished sum as the factor 2^(-lo);
+//   scalar  one thread, fp64: logp, rho, clipped surrogate, KL term, the row factor g_t, and the
+//         row's weighted loss term into the workspace;
+//   grad  the row a third time (L2): write bf16(g_t (onehot - softmax)).  Rows whose g_t is exactly
+//         0 (masked, or clipped with no KL term) are written as zeros without being re-read.
+// No sweep has a data-dependent branch except at the one vector holding the excluded maximum.
 // Loss reduction: a single CTA sums the chunk's per-row terms in a fixed order (deterministic).
 
 #include <cuda_bf16.h>
@@ -23,15 +24,15 @@
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kBatch = 4;          // 128-bit loads in flight per thread
 
 struct RowShared {
-    float red_f[32];
+    unsigned long long red_k[32];
     double red_d[32];
-    int red_i[32];
     float row_max;
-    double zprime;      // sum over the row of e^(x - max), one instance of the maximum excluded
-    int nmax_threads;
-    float coef;         // -g_t / Z
+    int max_pos;        // position code of the first instance of the maximum
+    double zprime;      // sum over the row of 2^(x log2e - ref), one instance of the maximum excluded
+    float coef;         // -g_t / Z (with the reference correction)
     float target;       // g_t (1 - p_token)
     int write_mode;     // 0: zeros, 1: gradient
     int token;
@@ -46,6 +47,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -56,100 +63,116 @@ __device__ __forceinline__ uint16_t to_bf16_bits(float v) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(v));
 }
 
-constexpr float kLn2 = 0.6931471805599453f;
+__device__ __forceinline__ uint4 ld_global_v4(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
 
-// Running (max, sum) of one thread: s = sum of 2^(x log2e - mxc) over the thread's elements except
-// one instance of the maximum, where the reference exponent mxc = fl(mx log2e) is an fp32 number in
-// its own right.  The fused multiply-add x*log2e - mxc is then rounded once, and the difference
-// lo = mx*log2e - mxc (exact in fp32, from one more fma) is applied to the finished sum as the
-// factor 2^(-lo), so the rounding of mx*log2e never enters the row's statistics.
-struct OnlineStat {
-    float mx;    // running maximum of the raw logits (-inf before the first element)
-    float mxc;   // fl(mx * log2(e))
-    float s;
-};
-
-// 2^(-lo) for lo = mx*log2e - fl(mx*log2e), |lo| < 2^-18: first-order expansion, fp64.
+// 2^(-lo) for lo = M*log2e - fl(M*log2e), |lo| < 2^-18: first-order expansion, fp64.
 __device__ __forceinline__ double ref_correction(float mx, float mxc) {
     return 1.0 - (double)fmaf(mx, kLog2e, -mxc) * 0.6931471805599453;
 }
 
-__device__ __forceinline__ void stat_add_slow(OnlineStat& st, const float* v, int cnt, float vmax) {
-    // A new maximum arrived: the old maximum becomes an ordinary element (worth 2^lo relative to
-    // the old reference), the sum moves to the new reference, and the first instance of the new
-    // maximum is left out of the sum.
-    const float ref = vmax * kLog2e;
-    if (st.mx != -INFINITY) {
-        const float lo_old = fmaf(st.mx, kLog2e, -st.mxc);
-        st.s = (st.s + fmaf(lo_old, kLn2, 1.0f)) * ex2_approx(st.mxc - ref);
-    }
-    st.mx = vmax;
-    st.mxc = ref;
+__device__ __forceinline__ float vec_max(const uint4& q) {
+    const uint32_t w = max_bf16x2(max_bf16x2(q.x, q.y), max_bf16x2(q.z, q.w));
+    return fmaxf(bf16_lo(w), bf16_hi(w));
+}
+
+__device__ __forceinline__ float vec_sum_ex2(const uint4& q, float ref) {
+    const float a = ex2_approx(fmaf(bf16_lo(q.x), kLog2e, -ref)) + ex2_approx(fmaf(bf16_hi(q.x), kLog2e, -ref));
+    const float b = ex2_approx(fmaf(bf16_lo(q.y), kLog2e, -ref)) + ex2_approx(fmaf(bf16_hi(q.y), kLog2e, -ref));
+    const float c = ex2_approx(fmaf(bf16_lo(q.z), kLog2e, -ref)) + ex2_approx(fmaf(bf16_hi(q.z), kLog2e, -ref));
+    const float d = ex2_approx(fmaf(bf16_lo(q.w), kLog2e, -ref)) + ex2_approx(fmaf(bf16_hi(q.w), kLog2e, -ref));
+    return (a + b) + (c + d);
+}
+
+// The vector that holds the excluded instance: every element but the first one equal to mx.
+__device__ __forceinline__ float ex2_unless(float x, float ref, float mx, bool& skipped) {
+    const bool skip = !skipped && x == mx;
+    skipped |= skip;
+    return skip ? 0.0f : ex2_approx(fmaf(x, kLog2e, -ref));
+}
+
+__device__ __noinline__ float vec_sum_ex2_excluding(uint4 q, float ref, float mx) {
     bool skipped = false;
-    for (int i = 0; i < cnt; ++i) {
-        if (!skipped && v[i] == vmax) { skipped = true; continue; }
-        st.s += ex2_approx(fmaf(v[i], kLog2e, -st.mxc));
-    }
+    float s = ex2_unless(bf16_lo(q.x), ref, mx, skipped);
+    s += ex2_unless(bf16_hi(q.x), ref, mx, skipped);
+    s += ex2_unless(bf16_lo(q.y), ref, mx, skipped);
+    s += ex2_unless(bf16_hi(q.y), ref, mx, skipped);
+    s += ex2_unless(bf16_lo(q.z), ref, mx, skipped);
+    s += ex2_unless(bf16_hi(q.z), ref, mx, skipped);
+    s += ex2_unless(bf16_lo(q.w), ref, mx, skipped);
+    s += ex2_unless(bf16_hi(q.w), ref, mx, skipped);
+    return s;
 }
 
-__device__ __forceinline__ void stat_add8(OnlineStat& st, const uint4& q) {
-    float v[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
-                  bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
-    const float vmax = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
-    if (vmax > st.mx) {
-        stat_add_slow(st, v, 8, vmax);
-    } else {
-        float a = 0.0f, b = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            a += ex2_approx(fmaf(v[i], kLog2e, -st.mxc));
-            b += ex2_approx(fmaf(v[i + 1], kLog2e, -st.mxc));
-        }
-        st.s += a + b;
-    }
+__device__ __forceinline__ uint4 grad_vec(const uint4& q, float coef, float ref) {
+    uint4 o;
+    o.x = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.x), kLog2e, -ref)),
+                      coef * ex2_approx(fmaf(bf16_hi(q.x), kLog2e, -ref)));
+    o.y = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.y), kLog2e, -ref)),
+                      coef * ex2_approx(fmaf(bf16_hi(q.y), kLog2e, -ref)));
+    o.z = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.z), kLog2e, -ref)),
+                      coef * ex2_approx(fmaf(bf16_hi(q.z), kLog2e, -ref)));
+    o.w = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.w), kLog2e, -ref)),
+                      coef * ex2_approx(fmaf(bf16_hi(q.w), kLog2e, -ref)));
+    return o;
 }
 
-__device__ __forceinline__ void stat_add1(OnlineStat& st, float v) {
-    if (v > st.mx) stat_add_slow(st, &v, 1, v);
-    else st.s += ex2_approx(fmaf(v, kLog2e, -st.mxc));
+// Replace element e (0..7) of a packed vector of eight bf16 values.
+__device__ __forceinline__ void patch_bf16(uint4& o, int e, uint16_t bits) {
+    const uint32_t shift = (e & 1) ? 16u : 0u;
+    const uint32_t keep = ~(0xffffu << shift), put = (uint32_t)bits << shift;
+    const int w = e >> 1;
+    o.x = w == 0 ? (o.x & keep) | put : o.x;
+    o.y = w == 1 ? (o.y & keep) | put : o.y;
+    o.z = w == 2 ? (o.z & keep) | put : o.z;
+    o.w = w == 3 ? (o.w & keep) | put : o.w;
 }
 
+// Block arg-max: the largest value, and among equal values the smallest position code.
 template <int BLOCK>
-__device__ __forceinline__ float block_max(float v, RowShared& sh) {
+__device__ __forceinline__ void block_argmax(float v, int pos, RowShared& sh) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(PODS_FULL_MASK, v, d));
-    if (lane == 0) sh.red_f[warp] = v;
-    __syncthreads();
-    if (warp == 0) {
-        float w = lane < BLOCK / 32 ? sh.red_f[lane] : -INFINITY;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) w = fmaxf(w, __shfl_xor_sync(PODS_FULL_MASK, w, d));
-        if (lane == 0) sh.row_max = w;
-    }
-    __syncthreads();
-    return sh.row_max;
-}
-
-template <int BLOCK>
-__device__ __forceinline__ void block_sum(double v, int c, RowShared& sh) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t u = __float_as_uint(v + 0.0f);                        // -0 -> +0
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);                // order-preserving bits
+    unsigned long long key = ((unsigned long long)u << 32) | (uint32_t)(0x7fffffff - pos);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
-        v += __shfl_xor_sync(PODS_FULL_MASK, v, d);
-        c += __shfl_xor_sync(PODS_FULL_MASK, c, d);
+        const unsigned long long o = __shfl_xor_sync(PODS_FULL_MASK, key, d);
+        key = o > key ? o : key;
     }
-    if (lane == 0) { sh.red_d[warp] = v; sh.red_i[warp] = c; }
+    if (lane == 0) sh.red_k[warp] = key;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long k = lane < BLOCK / 32 ? sh.red_k[lane] : 0ull;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(PODS_FULL_MASK, k, d);
+            k = o > k ? o : k;
+        }
+        if (lane == 0) {
+            const uint32_t o = (uint32_t)(k >> 32);
+            sh.row_max = __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+            sh.max_pos = 0x7fffffff - (int)(uint32_t)(k & 0xffffffffu);
+        }
+    }
+    __syncthreads();
+}
+
+template <int BLOCK>
+__device__ __forceinline__ void block_sum(double v, RowShared& sh) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(PODS_FULL_MASK, v, d);
+    if (lane == 0) sh.red_d[warp] = v;
     __syncthreads();
     if (warp == 0) {
         double w = lane < BLOCK / 32 ? sh.red_d[lane] : 0.0;
-        int k = lane < BLOCK / 32 ? sh.red_i[lane] : 0;
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            w += __shfl_xor_sync(PODS_FULL_MASK, w, d);
-            k += __shfl_xor_sync(PODS_FULL_MASK, k, d);
-        }
-        if (lane == 0) { sh.zprime = w; sh.nmax_threads = k; }
+        for (int d = 16; d > 0; d >>= 1) w += __shfl_xor_sync(PODS_FULL_MASK, w, d);
+        if (lane == 0) sh.zprime = w;
     }
     __syncthreads();
 }
@@ -194,6 +217,8 @@ grpo_loss_rows_kernel(const RowArgs a) {
     const int tid = threadIdx.x;
     const int V = a.V;
     const int nvec = a.vec_ok ? V / 8 : 0;
+    const int tail0 = nvec * 8;
+    // Position codes: vector v -> v, tail element e -> nvec + (e - tail0).
 
     for (int64_t t = blockIdx.x; t < a.T; t += gridDim.x) {
         const uint16_t* row = a.logits + t * a.ldl;
@@ -208,24 +233,56 @@ grpo_loss_rows_kernel(const RowArgs a) {
             x_tok = __uint_as_float((uint32_t)row[tok] << 16);   // read before anything is written in place
         }
 
-        // ---- pass 1: per-thread running maximum and sum -------------------------------------
-        OnlineStat st = {-INFINITY, -INFINITY, 0.0f};
-        for (int v = tid; v < nvec; v += BLOCK) stat_add8(st, row4[v]);
-        for (int v = nvec * 8 + tid; v < V; v += BLOCK) stat_add1(st, __uint_as_float((uint32_t)row[v] << 16));
-
-        const float mx = block_max<BLOCK>(st.mx, sh);
-        double contrib = 0.0;
-        int is_max = 0;
-        if (st.mx != -INFINITY) {
-            const double s_true = (double)st.s * ref_correction(st.mx, st.mxc);
-            if (st.mx == mx) { contrib = s_true; is_max = 1; }
-            else contrib = (s_true + 1.0) * (double)ex2_approx((st.mx - mx) * kLog2e);
+        // ---- sweep 1: maximum and where it is ----------------------------------------------
+        float m_t = -INFINITY;
+        int pos_t = 0x7fffffff;
+        for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
+            uint4 q[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int v = v0 + j * BLOCK;
+                q[j] = v < nvec ? ld_global_v4(row4 + v) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const float vm = vec_max(q[j]);
+                if (vm > m_t) { m_t = vm; pos_t = v0 + j * BLOCK; }
+            }
         }
-        block_sum<BLOCK>(contrib, is_max, sh);
+        for (int e = tail0 + tid; e < V; e += BLOCK) {
+            const float x = __uint_as_float((uint32_t)row[e] << 16);
+            if (x > m_t) { m_t = x; pos_t = nvec + (e - tail0); }
+        }
+        block_argmax<BLOCK>(m_t, pos_t, sh);
+        const float mx = sh.row_max;
+        const int excl = sh.max_pos;
+        const float ref = mx * kLog2e;
+
+        // ---- sweep 2: sum of exponentials, one instance of the maximum left out ---------------
+        float s_t = 0.0f;
+        for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
+            uint4 q[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int v = v0 + j * BLOCK;
+                q[j] = v < nvec ? ld_global_v4(row4 + v) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                if (v0 + j * BLOCK == excl) s_t += vec_sum_ex2_excluding(q[j], ref, mx);
+                else s_t += vec_sum_ex2(q[j], ref);                  // padding is -inf: adds 0
+            }
+        }
+        for (int e = tail0 + tid; e < V; e += BLOCK) {
+            const float x = __uint_as_float((uint32_t)row[e] << 16);
+            if (nvec + (e - tail0) != excl) s_t += ex2_approx(fmaf(x, kLog2e, -ref));
+        }
+        block_sum<BLOCK>((double)s_t, sh);
 
         // ---- scalar terms of the row (one thread, fp64) ---------------------------------------
         if (tid == 0) {
-            const double zp = sh.zprime + (double)(sh.nmax_threads - 1);   // all but one instance of the max
+            const double corr = ref_correction(mx, ref);
+            const double zp = sh.zprime * corr;                    // sum over all but one instance of the max
             const double Z = 1.0 + zp;
             const double logp = ((double)x_tok - (double)mx) - log1p(zp);
             const int64_t i = find_rollout(a.cu_seqlens, a.M, a.row0 + t);
@@ -248,47 +305,43 @@ grpo_loss_rows_kernel(const RowArgs a) {
             const double one_minus_p = (x_tok == mx) ? zp / Z : -expm1(logp);
             a.logp[t] = (float)logp;
             a.row_loss[t] = (w != 0.0) ? w * loss : 0.0;    // a masked row adds nothing, whatever its inputs
-            sh.coef = (float)(-g / Z * ref_correction(mx, mx * kLog2e));   // pass 2 uses fl(mx log2e) again
+            sh.coef = (float)(-g / Z * corr);
             sh.target = (float)(g * one_minus_p);
             sh.write_mode = (g != 0.0) ? 1 : 0;
         }
         __syncthreads();
 
-        // ---- pass 2: the gradient row ---------------------------------------------------------
+        // ---- sweep 3: the gradient row --------------------------------------------------------
         const int tok = sh.token;
+        uint4* d4 = reinterpret_cast<uint4*>(drow);
         if (sh.write_mode == 0) {
             const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            uint4* d4 = reinterpret_cast<uint4*>(drow);
             for (int v = tid; v < nvec; v += BLOCK) __stcs(d4 + v, z);
-            for (int v = nvec * 8 + tid; v < V; v += BLOCK) drow[v] = 0;
+            for (int e = tail0 + tid; e < V; e += BLOCK) drow[e] = 0;
         } else {
             const float coef = sh.coef;
-            const float mxc = mx * kLog2e;
             const uint16_t target_bits = to_bf16_bits(sh.target);
-            uint4* d4 = reinterpret_cast<uint4*>(drow);
             const int tok_vec = tok >> 3;
-            for (int v = tid; v < nvec; v += BLOCK) {
-                const uint4 q = row4[v];
-                uint4 o;
-                o.x = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.x), kLog2e, -mxc)),
-                                  coef * ex2_approx(fmaf(bf16_hi(q.x), kLog2e, -mxc)));
-                o.y = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.y), kLog2e, -mxc)),
-                                  coef * ex2_approx(fmaf(bf16_hi(q.y), kLog2e, -mxc)));
-                o.z = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.z), kLog2e, -mxc)),
-                                  coef * ex2_approx(fmaf(bf16_hi(q.z), kLog2e, -mxc)));
-                o.w = pack_bf16x2(coef * ex2_approx(fmaf(bf16_lo(q.w), kLog2e, -mxc)),
-                                  coef * ex2_approx(fmaf(bf16_hi(q.w), kLog2e, -mxc)));
-                if (v == tok_vec) {
-                    uint32_t* ow = &o.x;
-                    const int e = tok & 7;
-                    const uint32_t shift = (e & 1) ? 16u : 0u;
-                    ow[e >> 1] = (ow[e >> 1] & ~(0xffffu << shift)) | ((uint32_t)target_bits << shift);
+            for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
+                uint4 q[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int v = v0 + j * BLOCK;
+                    if (v < nvec) q[j] = ld_global_v4(row4 + v);
                 }
-                __stcs(d4 + v, o);
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int v = v0 + j * BLOCK;
+                    if (v < nvec) {
+                        uint4 o = grad_vec(q[j], coef, ref);
+                        if (v == tok_vec) patch_bf16(o, tok & 7, target_bits);
+                        __stcs(d4 + v, o);
+                    }
+                }
             }
-            for (int v = nvec * 8 + tid; v < V; v += BLOCK) {
-                const float x = __uint_as_float((uint32_t)row[v] << 16);
-                drow[v] = (v == tok) ? target_bits : to_bf16_bits(coef * ex2_approx(fmaf(x, kLog2e, -mxc)));
+            for (int e = tail0 + tid; e < V; e += BLOCK) {
+                const float x = __uint_as_float((uint32_t)row[e] << 16);
+                drow[e] = (e == tok) ? target_bits : to_bf16_bits(coef * ex2_approx(fmaf(x, kLog2e, -ref)));
             }
         }
         __syncthreads();     // sh is reused by the next row

@@ -44,6 +44,11 @@ WORKLOADS = {
     "c2_qwen_vocab": Workload("c2_qwen_vocab", G=8, n=64, m=16, rewards="bernoulli_beta", seed=1, V=151936,
                               len_kind="uniform", len_lo=64, len_hi=512, logit_sigma=3.0,
                               spike=8.0, spike_frac=0.3),
+    # one prompt group of config 2 (about 4.6k kept tokens, 1.4 GB of logits): small enough for a
+    # many-pass profiler capture, still far larger than L2
+    "c2_profile": Workload("c2_profile", G=1, n=64, m=16, rewards="bernoulli_beta", seed=1, V=151936,
+                           len_kind="uniform", len_lo=64, len_hi=512, logit_sigma=3.0,
+                           spike=8.0, spike_frac=0.3),
     "c3_select_mixed": Workload("c3_select_mixed", G=65536, n=32, m=8, rewards="mixed", seed=2),
     "c4_select_ties": Workload("c4_select_ties", G=16384, n=512, m=128, rewards="ternary", seed=3),
     "c5_large_loss": Workload("c5_large_loss", G=16, n=64, m=16, rewards="bernoulli_beta", seed=4, V=151936,
