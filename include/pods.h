@@ -44,6 +44,8 @@ typedef enum {
 #define PODS_STATUS_CAPACITY         0x4u  /* pods_compact: T exceeded T_cap (the excess was not written),
                                               or a length exceeded src_ld (it was cut to src_ld)          */
 #define PODS_STATUS_NEG_LENGTH       0x8u  /* pods_compact: a negative length was treated as 0            */
+#define PODS_STATUS_TIMEOUT          0x10u /* a bounded wait inside a kernel ran out (asynchronous copy never
+                                              completed); the results of that call are not valid           */
 
 /* Down-sampling rules D(o, r; m) of Section 3.2 / 3.3. */
 typedef enum {

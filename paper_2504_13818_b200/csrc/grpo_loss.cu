@@ -16,14 +16,12 @@
 // No sweep has a data-dependent branch except at the one vector holding the excluded maximum.
 // Loss reduction: a single CTA sums the chunk's per-row terms in a fixed order (deterministic).
 
-#include <cuda_bf16.h>
-#include <math.h>
+#include "grpo_loss_common.cuh"
 
-#include "pods_common.cuh"
+using namespace pods_loss;
 
 namespace {
 
-constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kBatch = 4;          // 128-bit loads in flight per thread
 
 struct RowShared {
@@ -38,45 +36,20 @@ struct RowShared {
     int token;
 };
 
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-__device__ __forceinline__ uint16_t to_bf16_bits(float v) {
-    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
-}
-
 __device__ __forceinline__ uint4 ld_global_v4(const uint4* p) {
     uint4 r;
     asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
 
-// 2^(-lo) for lo = M*log2e - fl(M*log2e), |lo| < 2^-18: first-order expansion, fp64.
-__device__ __forceinline__ double ref_correction(float mx, float mxc) {
-    return 1.0 - (double)fmaf(mx, kLog2e, -mxc) * 0.6931471805599453;
-}
-
-__device__ __forceinline__ float vec_max(const uint4& q) {
-    const uint32_t w = max_bf16x2(max_bf16x2(q.x, q.y), max_bf16x2(q.z, q.w));
-    return fmaxf(bf16_lo(w), bf16_hi(w));
+// One batch of kBatch vectors, BLOCK apart, starting at vector v0 (missing ones read as -inf).
+template <int BLOCK>
+__device__ __forceinline__ void load_batch(uint4 (&q)[kBatch], const uint4* row4, int v0, int nvec) {
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+        const int v = v0 + j * BLOCK;
+        q[j] = v < nvec ? ld_global_v4(row4 + v) : make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+    }
 }
 
 __device__ __forceinline__ float vec_sum_ex2(const uint4& q, float ref) {
@@ -120,24 +93,11 @@ __device__ __forceinline__ uint4 grad_vec(const uint4& q, float coef, float ref)
     return o;
 }
 
-// Replace element e (0..7) of a packed vector of eight bf16 values.
-__device__ __forceinline__ void patch_bf16(uint4& o, int e, uint16_t bits) {
-    const uint32_t shift = (e & 1) ? 16u : 0u;
-    const uint32_t keep = ~(0xffffu << shift), put = (uint32_t)bits << shift;
-    const int w = e >> 1;
-    o.x = w == 0 ? (o.x & keep) | put : o.x;
-    o.y = w == 1 ? (o.y & keep) | put : o.y;
-    o.z = w == 2 ? (o.z & keep) | put : o.z;
-    o.w = w == 3 ? (o.w & keep) | put : o.w;
-}
-
 // Block arg-max: the largest value, and among equal values the smallest position code.
 template <int BLOCK>
 __device__ __forceinline__ void block_argmax(float v, int pos, RowShared& sh) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t u = __float_as_uint(v + 0.0f);                        // -0 -> +0
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);                // order-preserving bits
-    unsigned long long key = ((unsigned long long)u << 32) | (uint32_t)(0x7fffffff - pos);
+    unsigned long long key = argmax_key(v, pos);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
         const unsigned long long o = __shfl_xor_sync(PODS_FULL_MASK, key, d);
@@ -153,9 +113,8 @@ __device__ __forceinline__ void block_argmax(float v, int pos, RowShared& sh) {
             k = o > k ? o : k;
         }
         if (lane == 0) {
-            const uint32_t o = (uint32_t)(k >> 32);
-            sh.row_max = __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
-            sh.max_pos = 0x7fffffff - (int)(uint32_t)(k & 0xffffffffu);
+            sh.row_max = argmax_key_value(k);
+            sh.max_pos = argmax_key_pos(k);
         }
     }
     __syncthreads();
@@ -177,41 +136,8 @@ __device__ __forceinline__ void block_sum(double v, RowShared& sh) {
     __syncthreads();
 }
 
-struct RowArgs {
-    const uint16_t* logits;
-    int64_t ldl;
-    const int32_t* tokens;
-    const float* old_logp;
-    const float* ref_logp;
-    const float* adv;
-    const double* seq_weight;
-    const int64_t* cu_seqlens;
-    int64_t M;
-    int64_t row0;
-    const uint8_t* mask;
-    int64_t T;
-    int32_t V;
-    float eps, beta, grad_scale;
-    float* logp;
-    uint16_t* dlogits;
-    int64_t ldd;
-    double* row_loss;      // workspace [T]: mask_t w_i loss_t
-    uint32_t* status;
-    int vec_ok;            // 16-byte aligned rows: 128-bit path
-};
-
-// Rollout of packed row r: the i with cu_seqlens[i] <= r < cu_seqlens[i+1].
-__device__ __forceinline__ int64_t find_rollout(const int64_t* cu, int64_t M, int64_t r) {
-    int64_t lo = 0, hi = M;            // invariant: cu[lo] <= r, answer in [lo, hi)
-    while (hi - lo > 1) {
-        const int64_t mid = (lo + hi) >> 1;
-        if (cu[mid] <= r) lo = mid; else hi = mid;
-    }
-    return lo;
-}
-
 template <int BLOCK>
-__global__ void __launch_bounds__(BLOCK)
+__global__ void __launch_bounds__(BLOCK, 2048 / BLOCK / 2)
 grpo_loss_rows_kernel(const RowArgs a) {
     __shared__ RowShared sh;
     const int tid = threadIdx.x;
@@ -234,19 +160,22 @@ grpo_loss_rows_kernel(const RowArgs a) {
         }
 
         // ---- sweep 1: maximum and where it is ----------------------------------------------
+        // (every sweep keeps the next batch of loads in flight while it works on the current one)
         float m_t = -INFINITY;
         int pos_t = 0x7fffffff;
-        for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
-            uint4 q[kBatch];
+        {
+            uint4 nxt[kBatch];
+            load_batch<BLOCK>(nxt, row4, tid, nvec);
+            for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
+                uint4 q[kBatch];
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int v = v0 + j * BLOCK;
-                q[j] = v < nvec ? ld_global_v4(row4 + v) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-            }
+                for (int j = 0; j < kBatch; ++j) q[j] = nxt[j];
+                if (v0 + kBatch * BLOCK < nvec) load_batch<BLOCK>(nxt, row4, v0 + kBatch * BLOCK, nvec);
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const float vm = vec_max(q[j]);
-                if (vm > m_t) { m_t = vm; pos_t = v0 + j * BLOCK; }
+                for (int j = 0; j < kBatch; ++j) {
+                    const float vm = vec_max(q[j]);
+                    if (vm > m_t) { m_t = vm; pos_t = v0 + j * BLOCK; }
+                }
             }
         }
         for (int e = tail0 + tid; e < V; e += BLOCK) {
@@ -260,17 +189,19 @@ grpo_loss_rows_kernel(const RowArgs a) {
 
         // ---- sweep 2: sum of exponentials, one instance of the maximum left out ---------------
         float s_t = 0.0f;
-        for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
-            uint4 q[kBatch];
+        {
+            uint4 nxt[kBatch];
+            load_batch<BLOCK>(nxt, row4, tid, nvec);
+            for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
+                uint4 q[kBatch];
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int v = v0 + j * BLOCK;
-                q[j] = v < nvec ? ld_global_v4(row4 + v) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-            }
+                for (int j = 0; j < kBatch; ++j) q[j] = nxt[j];
+                if (v0 + kBatch * BLOCK < nvec) load_batch<BLOCK>(nxt, row4, v0 + kBatch * BLOCK, nvec);
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                if (v0 + j * BLOCK == excl) s_t += vec_sum_ex2_excluding(q[j], ref, mx);
-                else s_t += vec_sum_ex2(q[j], ref);                  // padding is -inf: adds 0
+                for (int j = 0; j < kBatch; ++j) {
+                    if (v0 + j * BLOCK == excl) s_t += vec_sum_ex2_excluding(q[j], ref, mx);
+                    else s_t += vec_sum_ex2(q[j], ref);              // padding is -inf: adds 0
+                }
             }
         }
         for (int e = tail0 + tid; e < V; e += BLOCK) {
@@ -282,32 +213,13 @@ grpo_loss_rows_kernel(const RowArgs a) {
         // ---- scalar terms of the row (one thread, fp64) ---------------------------------------
         if (tid == 0) {
             const double corr = ref_correction(mx, ref);
-            const double zp = sh.zprime * corr;                    // sum over all but one instance of the max
-            const double Z = 1.0 + zp;
-            const double logp = ((double)x_tok - (double)mx) - log1p(zp);
-            const int64_t i = find_rollout(a.cu_seqlens, a.M, a.row0 + t);
-            const bool live = a.mask == nullptr || a.mask[t] != 0;
-            const double w = live ? a.seq_weight[i] : 0.0;
-            const double adv = (double)a.adv[i];
-            const double eps = (double)a.eps, beta = (double)a.beta;
-            const double rho = exp(logp - (double)a.old_logp[t]);
-            const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
-            const double s1 = rho * adv, s2 = clipped * adv;
-            double loss = -(s1 < s2 ? s1 : s2);
-            double dl = (s1 <= s2) ? -adv * rho : 0.0;
-            if (a.ref_logp != nullptr && beta != 0.0) {
-                const double d = (double)a.ref_logp[t] - logp;
-                const double ed = exp(d);
-                loss += beta * (ed - d - 1.0);
-                dl += beta * (1.0 - ed);
-            }
-            const double g = (w != 0.0) ? (double)a.grad_scale * w * dl : 0.0;
-            const double one_minus_p = (x_tok == mx) ? zp / Z : -expm1(logp);
-            a.logp[t] = (float)logp;
-            a.row_loss[t] = (w != 0.0) ? w * loss : 0.0;    // a masked row adds nothing, whatever its inputs
-            sh.coef = (float)(-g / Z * corr);
-            sh.target = (float)(g * one_minus_p);
-            sh.write_mode = (g != 0.0) ? 1 : 0;
+            const RowInputs in = load_row_inputs(a, t);
+            const RowScalars r = row_scalars(a, in, x_tok, mx, sh.zprime * corr);
+            a.logp[t] = (float)r.logp;
+            a.row_loss[t] = r.weighted_loss;
+            sh.coef = (float)(-r.g / r.Z * corr);
+            sh.target = (float)(r.g * r.one_minus_p);
+            sh.write_mode = (r.g != 0.0) ? 1 : 0;
         }
         __syncthreads();
 
@@ -322,13 +234,13 @@ grpo_loss_rows_kernel(const RowArgs a) {
             const float coef = sh.coef;
             const uint16_t target_bits = to_bf16_bits(sh.target);
             const int tok_vec = tok >> 3;
+            uint4 nxt[kBatch];
+            load_batch<BLOCK>(nxt, row4, tid, nvec);
             for (int v0 = tid; v0 < nvec; v0 += kBatch * BLOCK) {
                 uint4 q[kBatch];
 #pragma unroll
-                for (int j = 0; j < kBatch; ++j) {
-                    const int v = v0 + j * BLOCK;
-                    if (v < nvec) q[j] = ld_global_v4(row4 + v);
-                }
+                for (int j = 0; j < kBatch; ++j) q[j] = nxt[j];
+                if (v0 + kBatch * BLOCK < nvec) load_batch<BLOCK>(nxt, row4, v0 + kBatch * BLOCK, nvec);
 #pragma unroll
                 for (int j = 0; j < kBatch; ++j) {
                     const int v = v0 + j * BLOCK;
@@ -420,8 +332,16 @@ extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* t
     a.vec_ok = pods_aligned(logits, 16) && pods_aligned(dlogits, 16) && ldl % 8 == 0 && ldd % 8 == 0;
 
     cudaStream_t s = pods_stream(stream);
-    constexpr int BLOCK = 1024;
-    const int64_t cap = (int64_t)pods_sm_count();
+    bool on_cluster_path = false;
+    const int rc_cluster = launch_grpo_loss_cluster(a, s, &on_cluster_path);
+    if (rc_cluster != PODS_OK) return rc_cluster;
+    if (on_cluster_path) {
+        loss_reduce_kernel<<<1, 1024, 0, s>>>(a.row_loss, T_chunk, loss_acc);
+        PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+        return PODS_OK;
+    }
+    constexpr int BLOCK = 512;
+    const int64_t cap = (int64_t)pods_sm_count() * 2;
     const int grid = (int)(T_chunk < cap ? T_chunk : cap);
     grpo_loss_rows_kernel<BLOCK><<<grid, BLOCK, 0, s>>>(a);
     PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());

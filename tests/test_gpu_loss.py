@@ -183,3 +183,53 @@ def test_whole_path_chained_on_its_own_outputs():
                                                w.eps, w.beta, cu, chunk_rows=500)
     torch.cuda.synchronize()
     _check(b, (float(loss.item()), logp.cpu().numpy(), dl.view(torch.uint16).cpu().numpy(), 0), want)
+
+
+# ---- rows large enough for the cluster-resident path (V >= 16384, V % 8 == 0, aligned) -----------
+
+@pytest.mark.parametrize("V,G,len_hi", [(16384, 6, 24),      # eight full segments; > 74 clusters' worth of rows
+                                        (20008, 2, 12),      # ragged last segment (2501 vectors over 8 CTAs)
+                                        (50000, 2, 10),
+                                        (151936, 1, 8)])     # the Qwen vocabulary
+def test_cluster_path_vocab_sizes(V, G, len_hi):
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=G, n=8, m=4, len_lo=4, len_hi=len_hi, seed=V % 1000)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    got = _gpu_loss(b)
+    _check(b, got, want)
+    again = _gpu_loss(b, in_place=True)
+    assert again[2].tobytes() == got[2].tobytes() and again[1].tobytes() == got[1].tobytes()
+
+
+def test_cluster_path_many_rows_per_cluster_masks_and_peaks():
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=16384, G=16, n=8, m=4, len_lo=8, len_hi=24, seed=77)
+    b = build_batch(w)
+    T = b["tokens"].shape[0]
+    assert T > 3 * 74                                   # several rows per resident cluster: buffers are reused
+    rng = np.random.default_rng(5)
+    b["mask"] = (rng.uniform(size=T) < 0.8).astype(np.uint8)
+    x = wl.bf16_bits_to_f32(b["logits"])
+    peak = rng.uniform(size=T) < 0.25                   # a quarter of the rows nearly certain of their token
+    x[peak, b["tokens"][peak]] += rng.uniform(12.0, 22.0, size=int(peak.sum())).astype(np.float32)
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
+    want = oracle_loss(b)
+    got = _gpu_loss(b, chunk_rows=300)
+    _check(b, got, want)
+    assert (got[2][b["mask"] == 0] == 0).all()
+    assert _gpu_loss(b, chunk_rows=300)[2].tobytes() == got[2].tobytes()      # run-to-run bit equality
+
+
+def test_cluster_path_token_in_every_segment_and_duplicate_maxima():
+    V = 16384
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=8, len_hi=8, seed=3, spike_frac=0.0)
+    b = build_batch(w)
+    T = b["tokens"].shape[0]
+    b["tokens"] = ((np.arange(T) * (V // 8) + 7 * np.arange(T)) % V).astype(np.int32)     # walks over the segments
+    x = wl.bf16_bits_to_f32(b["logits"])
+    x[0, [5, 9000, 16000]] = 14.0                       # the maximum three times, in different segments
+    x[1, b["tokens"][1]] = 15.0
+    x[1, (b["tokens"][1] + 1) % V] = 15.0               # the maximum twice in one vector, the token being one
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
+    _check(b, _gpu_loss(b), oracle_loss(b))
