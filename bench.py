@@ -168,7 +168,8 @@ class Batch:
         self.chunk = min(w.chunk_rows, T)
         self.ws = torch.empty(binding.grpo_loss_chunk_workspace_bytes(self.chunk), dtype=torch.uint8, device=dev)
         self.n_chunks = (T + self.chunk - 1) // self.chunk
-        self.launches_per_step = 1 + 2 + 1 + 1 + 2 * self.n_chunks + 1   # select, compact(2), zero, weights, chunks, finalize
+        # select, compact (scan + gather), weights, per chunk (row records + fused loss + reduction), finalize
+        self.launches_per_step = 1 + 2 + 1 + 3 * self.n_chunks + 1
         self.loss_events = []
 
     def step(self, record=False):
@@ -238,7 +239,7 @@ def cpu_baseline(batch, budget_rows=None):
     mask = np.ones(T, np.uint8)
     t0 = time.perf_counter()
     sw = oracle.seq_weights(mask, cu)
-    repeats = 3 if w.V > 50000 else 1           # the same rows again: ~20 core-seconds in all at V=151936
+    repeats = 24 if w.V > 50000 else 1          # the same rows again: about ten seconds of CPU work at V=151936
     for _ in range(repeats):
         out = oracle.grpo_rows(lg, toks[:rows], old, ref, sel["adv"].astype(np.float32).reshape(-1), sw,
                                seq_of_row[:rows], mask[:rows], w.eps, w.beta, want_dlogits=True)
@@ -304,7 +305,7 @@ def run_ours(args):
     bytes_per_token = 4 * w.V + 21
     achieved = bytes_per_token * batch.chunk / (per_launch_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
-    roofline = {"kernel": "grpo_loss_rows_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+    roofline = {"kernel": "grpo_loss_cluster_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
                 "frac_of_nominal_8TBps": achieved / 8000.0, "traffic": None,
                 "bytes_per_launch": bytes_per_token * batch.chunk, "ms_per_launch": per_launch_ms,
@@ -340,29 +341,25 @@ def run_ours(args):
 
 
 def run_e2e(batch, args):
-    """The same step through the host-buffer entry point: inputs in pinned host memory, results read back."""
-    from paper_2504_13818_b200 import binding
-    if not hasattr(binding, "pods_step_host"):
-        return None
-    return binding_e2e(batch, args)
-
-
-def binding_e2e(batch, args):
+    """The same step through the host-buffer entry point (pods_host_step_run): every input starts in
+    pinned host memory, every copy is inside the timed region, loss / logp / idx / adv are read back."""
     from paper_2504_13818_b200 import binding
     w = batch.w
     host = binding.HostStep(w.G, w.n, w.m, batch.src_tokens_h.shape[1], batch.T, w.V, chunk_rows=2048)
     host.set_inputs(batch.rewards_h, batch.lengths_h, batch.src_tokens_h, batch.src_old_h, batch.src_ref_h,
                     batch.logits)
-    steps = max(2, min(args.steps, 3))
-    for _ in range(1):
-        host.run(w.eps, w.beta)
+    steps = max(2, min(args.steps, 5))
+    host.run(w.eps, w.beta)
     t0 = time.perf_counter()
     for _ in range(steps):
         host.run(w.eps, w.beta)
     dt = time.perf_counter() - t0
-    return {"value": batch.T * steps / dt, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes,
-            "d2h_bytes_per_step": host.d2h_bytes, "steps": steps, "ms_per_step": dt / steps * 1e3,
-            "loss": host.loss()}
+    out = {"value": batch.T * steps / dt, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes,
+           "d2h_bytes_per_step": host.d2h_bytes, "steps": steps, "ms_per_step": dt / steps * 1e3,
+           "h2d_GBps": host.h2d_bytes / (dt / steps) / 1e9, "loss": host.loss(),
+           "note": "dlogits stays on the device (pods_host_step_dlogits)"}
+    host.close()
+    return out
 
 
 # --------------------------------------------------------------------------------------------

@@ -7,7 +7,8 @@
  * Conventions for every call
  *   - Pointers marked [dev] are device pointers on the current CUDA device, [host] are host
  *     pointers.  The caller owns every buffer; the library allocates no device memory and
- *     keeps no state between calls (except pods_step_host, which says what it allocates).
+ *     keeps no state between calls (except pods_host_step_*, which says what it allocates, and
+ *     grpo_loss_chunk_static, which says what it holds).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
  *     enqueue work and return; outputs are valid once the stream has reached that point.
  *   - The return value is a pods_status.  Errors that the host can see (sizes, null or
@@ -166,9 +167,10 @@ int grpo_loss_fwd_bwd(const void* logits, int64_t ldl, const int32_t* tokens, co
  * after start-up, a process whose allocator is frozen while a profiler or checkpointer is attached.
  * (The paper has no counterpart; this is a packaging variant of the same computation.)
  *
- * The per-row loss terms that grpo_loss_chunk keeps in the caller's workspace are kept here in a
- * fixed array inside the library image: grpo_loss_chunk_static_max_rows() rows (16384) of fp64,
- * 128.5 KB, resident on every GPU that loads the library until the process exits.  The call itself
+ * What grpo_loss_chunk keeps in the caller's workspace (per row: its loss term and a 32-byte record
+ * of its scalar inputs) is kept here in a fixed array inside the library image, sized for
+ * grpo_loss_chunk_static_max_rows() rows (16384): 640.5 KB, resident on every GPU that loads the
+ * library until the process exits.  The call itself
  * calls no cudaMalloc, cudaFree or allocating library routine.  Same arguments, outputs and status
  * bits as grpo_loss_chunk, minus workspace/workspace_bytes.
  *
@@ -177,7 +179,7 @@ int grpo_loss_fwd_bwd(const void* logits, int64_t ldl, const int32_t* tokens, co
  *   - The first call on each device looks up the array's device address (a host-side runtime query,
  *     with that device current) and remembers it; make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the last call's contents.  Nothing in it
- *     needs clearing: each call overwrites the T_chunk slots it later sums.  Two calls that can run
+ *     needs clearing: each call overwrites the T_chunk slots it later reads.  Two calls that can run
  *     at the same time on the GPU (different streams, no ordering between them) race on it and give
  *     a wrong loss_acc; order them, or use grpo_loss_chunk with separate workspaces.
  */
@@ -191,6 +193,42 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
 
 /* Convert the fp64 accumulator of grpo_loss_chunk calls to the fp32 loss.  Both [dev]. */
 int grpo_loss_finalize(const double* loss_acc, float* loss, void* stream);
+
+/*
+ * pods_host_step - the whole path of one training batch for callers whose data is in HOST memory:
+ * D(o, r; m) and a_{S,i} (Sections 3.2-3.3), concatenation of the kept rollouts (text after
+ * Algorithm 1) and L_PODS with its gradient (Section 3.2), i.e. pods_select -> pods_compact ->
+ * grpo_seq_weights -> grpo_loss_chunk per chunk -> grpo_loss_finalize, with the copies around them.
+ *
+ * pods_host_step_create allocates, on the current device, every buffer the step needs (the only
+ * calls of this library that allocate): rollout storage for G*n rollouts of src_ld tokens, packed
+ * per-token arrays of T_cap entries, two staging buffers of chunk_rows x V bf16 logits, the
+ * gradient [T_cap, V] bf16, the loss workspace, two streams and four events.  V % 8 == 0 is
+ * required.  pods_host_step_destroy frees them.  One object serves one thread at a time.
+ *
+ * pods_host_step_run, all pointers [host] (pinned memory makes the copies asynchronous):
+ *   rewards fp32 [G,n]; lengths int32 [G*n]; src_tokens int32, src_old, src_ref fp32 [G*n, src_ld]
+ *   (src_ref may be NULL iff beta == 0); logits bf16 [T_logits, V], densely packed: the rows of the
+ *   kept rollouts in kept order - the caller must know which rollouts the rule keeps (it does when the
+ *   logits come from a forward pass over the kept rollouts only); if the device finds another T the
+ *   call stops after the compaction, *T_out holds the device's T and PODS_ERR_INVALID_ARG is returned.
+ *   Outputs: loss_out fp32 [1]; logp_out fp32 [T] or NULL; idx_out int32 [G,m] or NULL; adv_out
+ *   fp32 [G,m] or NULL; T_out, status_out (the device status word) or NULL.
+ * The logits are uploaded chunk by chunk on a second stream while the previous chunk's loss kernel
+ * runs.  dlogits [T, V] (row pitch V) stays on the device for the backward pass that consumes it:
+ * pods_host_step_dlogits returns its [dev] address, valid until the next run or destroy.  The call
+ * returns when every result is in place.
+ */
+typedef struct pods_host_step pods_host_step;
+int pods_host_step_create(int64_t G, int32_t n, int32_t m, int64_t src_ld, int64_t T_cap, int32_t V,
+                          int64_t chunk_rows, pods_host_step** out);
+int pods_host_step_run(pods_host_step* step, const float* rewards, const int32_t* lengths,
+                       const int32_t* src_tokens, const float* src_old, const float* src_ref, const void* logits,
+                       int64_t T_logits, float eps, float beta, int32_t rule, uint64_t seed, uint32_t flags,
+                       float* loss_out, float* logp_out, int32_t* idx_out, float* adv_out, int64_t* T_out,
+                       uint32_t* status_out);
+void* pods_host_step_dlogits(pods_host_step* step);
+int pods_host_step_destroy(pods_host_step* step);
 
 #ifdef __cplusplus
 }

@@ -39,6 +39,11 @@ SIGNATURES = {
     "grpo_loss_fwd_bwd": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i32, _f32, _f32, _i64,
                                     _p, _p, _p, _i64, _p, _sz, _p, _p]),
     "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
+    "pods_host_step_create": (C.c_int, [_i64, _i32, _i32, _i64, _i64, _i32, _i64, _p]),
+    "pods_host_step_run": (C.c_int, [_p, _p, _p, _p, _p, _p, _p, _i64, _f32, _f32, _i32, _u64, _u32,
+                                     _p, _p, _p, _p, _p, _p]),
+    "pods_host_step_dlogits": (_p, [_p]),
+    "pods_host_step_destroy": (C.c_int, [_p]),
 }
 
 _lib = None
@@ -264,3 +269,77 @@ def grpo_loss_fwd_bwd(logits, tokens, old_logp, ref_logp, adv, mask, eps, beta, 
                                   _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_loss_fwd_bwd")
     return loss, logp, dlogits
+
+
+class HostStep:
+    """pods_host_step_*: the whole path for inputs in host memory (pinned torch CPU tensors).
+
+    Marshalling only: ``set_inputs`` keeps references to the caller's host tensors (and pins a host
+    copy of the logits if they are handed over as a device tensor), ``run`` passes their addresses to
+    pods_host_step_run, which does every copy and every step."""
+
+    def __init__(self, G, n, m, src_ld, T_cap, V, chunk_rows=2048):
+        self.G, self.n, self.m, self.src_ld, self.T_cap, self.V = G, n, m, src_ld, T_cap, V
+        self._h = C.c_void_p()
+        _check(load().pods_host_step_create(G, n, m, src_ld, T_cap, V, chunk_rows, C.byref(self._h)),
+               "pods_host_step_create")
+        pin = dict(pin_memory=True)
+        self.loss_h = torch.zeros(1, dtype=torch.float32, **pin)
+        self.logp_h = torch.zeros(T_cap, dtype=torch.float32, **pin)
+        self.idx_h = torch.zeros((G, m), dtype=torch.int32, **pin)
+        self.adv_h = torch.zeros((G, m), dtype=torch.float32, **pin)
+        self.T_h = C.c_int64(0)
+        self.status_h = C.c_uint32(0)
+        self._in = None
+
+    @staticmethod
+    def _host(a, dtype):
+        t = a if isinstance(a, torch.Tensor) else torch.from_numpy(a)
+        t = t.to(dtype=dtype, device="cpu").contiguous()
+        return t if t.is_pinned() else t.pin_memory()
+
+    def set_inputs(self, rewards, lengths, src_tokens, src_old, src_ref, logits):
+        """Host arrays (numpy or CPU tensors) of one batch; ``logits`` [T,V] bf16 (a device tensor is copied to pinned host memory)."""
+        lg = logits.detach().to("cpu") if logits.is_cuda else logits
+        lg = lg.contiguous()
+        self._in = (self._host(rewards, torch.float32), self._host(lengths, torch.int32),
+                    self._host(src_tokens, torch.int32), self._host(src_old, torch.float32),
+                    None if src_ref is None else self._host(src_ref, torch.float32),
+                    lg if lg.is_pinned() else lg.pin_memory())
+        r, l, st, so, sr, lg = self._in
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self._in if t is not None)
+        self.d2h_bytes = 4 + 8 + 4 + 4 * lg.shape[0] + 8 * self.G * self.m
+
+    def run(self, eps, beta, rule=RULE_MAXVAR, seed=0, flags=0):
+        r, l, st, so, sr, lg = self._in
+        rc = load().pods_host_step_run(self._h, r.data_ptr(), l.data_ptr(), st.data_ptr(), so.data_ptr(),
+                                       None if sr is None else sr.data_ptr(), lg.data_ptr(), lg.shape[0], eps, beta,
+                                       rule, seed, flags, self.loss_h.data_ptr(), self.logp_h.data_ptr(),
+                                       self.idx_h.data_ptr(), self.adv_h.data_ptr(), C.byref(self.T_h),
+                                       C.byref(self.status_h))
+        _check(rc, "pods_host_step_run")
+        return float(self.loss_h[0])
+
+    def loss(self) -> float:
+        return float(self.loss_h[0])
+
+    def dlogits(self):
+        """The gradient [T,V] bf16 left on the device by the last run (a view; valid until the next run)."""
+        T = int(self.T_h.value)
+        ptr = load().pods_host_step_dlogits(self._h)
+        # wrap the device pointer without copying: torch has no public from-pointer constructor, so go through
+        # the CUDA array interface
+        class _Arr:
+            __cuda_array_interface__ = {"shape": (T, self.V), "typestr": "<u2", "data": (int(ptr), False), "version": 2}
+        return torch.as_tensor(_Arr(), device="cuda").view(torch.bfloat16)
+
+    def close(self):
+        if self._h:
+            load().pods_host_step_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -285,7 +285,7 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 extern "C" size_t grpo_loss_chunk_workspace_bytes(int64_t T_chunk) {
     if (T_chunk < 0) return 0;
-    return align_up((size_t)T_chunk * sizeof(double), 256) + 256;
+    return align_up((size_t)T_chunk * sizeof(double), 256) + align_up((size_t)T_chunk * sizeof(RowPrep), 256) + 256;
 }
 
 extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* tokens, const float* old_logp,
@@ -328,6 +328,7 @@ extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* t
     a.dlogits = static_cast<uint16_t*>(dlogits);
     a.ldd = ldd;
     a.row_loss = static_cast<double*>(workspace);
+    a.prep = reinterpret_cast<RowPrep*>(static_cast<unsigned char*>(workspace) + align_up((size_t)T_chunk * sizeof(double), 256));
     a.status = status;
     a.vec_ok = pods_aligned(logits, 16) && pods_aligned(dlogits, 16) && ldl % 8 == 0 && ldd % 8 == 0;
 
@@ -408,7 +409,7 @@ extern "C" int grpo_loss_finalize(const double* loss_acc, float* loss, void* str
 namespace {
 
 // One fp64 slot per row of the largest chunk, plus the pad the workspace size formula asks for.
-constexpr size_t kStaticScratchBytes = (size_t)PODS_STATIC_CHUNK_ROWS * sizeof(double) + 512;
+constexpr size_t kStaticScratchBytes = (size_t)PODS_STATIC_CHUNK_ROWS * (sizeof(double) + sizeof(RowPrep)) + 512;
 static __device__ __align__(256) unsigned char g_static_row_loss[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;

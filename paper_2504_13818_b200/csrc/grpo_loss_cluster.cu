@@ -1,30 +1,45 @@
-// grpo_loss, cluster-resident rows: the fast path of the GRPO-PODS loss + gradient kernel.
+// grpo_loss, cluster-resident rows: the fast path of the GRPO-PODS loss + gradient kernel
+// (L_PODS of Section 3.2 and its derivative with respect to the bf16 logits).
 //
-// A thread-block cluster of CL CTAs owns one row of bf16 logits at a time; CTA r keeps the r-th
-// segment of the row in its shared memory from the moment it is loaded until its gradient has been
-// stored, so HBM sees exactly one read and one write per element and every other access is to
-// shared memory.  Several clusters are resident per SM group, each in a different phase, so that
-// the DRAM-bound load, the MUFU-bound sum and the store overlap.  Per row and CTA:
+// A thread-block cluster of CL CTAs owns one row of logits at a time; CTA r keeps the r-th segment
+// of the row in its shared memory from the moment it is loaded until its gradient has been stored,
+// so HBM sees exactly one read and one write per element and every other access is to shared
+// memory.  A CTA is eight consumer warps, one producer warp and one exchange warp that meet only
+// through mbarriers, over a ring of NS segment buffers; no warp ever waits at a CTA-wide barrier.
 //
-//   load    one thread issues bulk asynchronous copies global -> shared (8 KB pieces counted on one
-//           mbarrier, never multicast) as soon as the previous row's store has finished reading the
-//           buffer; another thread fetches the row's scalar inputs meanwhile;
-//   max     packed bf16x2 maxima of the segment; block arg-max (m_r and its first position);
-//   sum     e = 2^(x log2e - ref_r), ref_r = fl(m_r log2e), once per element: summed in fp32 per
-//           thread / fp64 across threads with that one instance of m_r left out (this keeps Z - 1
-//           accurate when one logit dominates), and bf16(e) written back in place;
-//   share   (m_r, position, sum_r) published in shared memory; ONE cluster barrier; warp 0 of
-//           every CTA reads the CL triples through distributed shared memory, combines them into
-//           the row maximum M and Z - 1, and evaluates the fp64 scalar terms with its lanes in
-//           parallel (redundantly per CTA: no second barrier);
-//   grad    in place: bf16(coef_r * e) by a packed bf16 fused multiply-add with coef_r split into
-//           two bf16 terms (coef_r folds in 2^(ref_r - M log2e)); the target entry is then
-//           overwritten with g (1 - p);
-//   store   one bulk asynchronous copy shared -> global of the whole segment.
+//   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
+//             pieces counted on the stage's `full` barrier, never multicast); as soon as the
+//             consumers report a stage `done` it loads the row NS ahead into it.
+//   consumer  warp w owns a fixed slice of the segment and is independent of the other warps:
+//       front(i)  the slice is read from shared memory ONCE into registers (IT vectors per lane);
+//                 max    packed bf16x2 maxima, warp arg-max -> m_w and the vector that holds its
+//                        first instance;
+//                 sum    e = 2^(x log2e - ref_w), ref_w = fl(m_w log2e), once per element, summed
+//                        in fp32 with that ONE instance of m_w left out (this keeps Z - 1 accurate
+//                        when one logit dominates), bf16(e) written back to shared memory in place;
+//                        (m_w, sum_w) is handed to the exchange warp;
+//       back(i-1) grad   bf16(coef_w * e) by packed bf16 multiply-adds with coef_w split into two
+//                        bf16 terms (coef_w folds in 2^(ref_w - M log2e)), the target entry replaced
+//                        by g (1 - p), stored straight to global memory with 128-bit streaming
+//                        stores; the warp then arrives on the stage's `done` barrier.
+//             front(i) runs before back(i-1), so the exchange of row i-1 has a whole sweep to finish.
+//             Shared memory sees 8 bytes of traffic per element (2 in, 2 read, 2 written, 2 read).
+//   exchange  for every row: writes the CTA's eight (m_w, sum_w) pairs into the slots it owns in
+//             every peer's shared memory, each as ONE 64-bit word that carries the row's tag, so
+//             that no fence or barrier crosses the cluster: a reader polls its 8 CL slots until all
+//             show the tag.  It then combines the pairs into the row maximum M and Z - 1, evaluates
+//             the fp64 scalar terms of the objective (three exponentials in one call on three
+//             lanes, no logarithm), publishes the eight coef_w, and only then (nobody waits for it)
+//             takes the logarithm for logp and the loss.
 //
-// The wait on the load's mbarrier is bounded: after kSpinLimit failed polls the CTA raises
-// PODS_STATUS_TIMEOUT and carries on with whatever is in the buffer, still taking part in every
-// barrier, so neither it nor its cluster peers can hang.
+// Every wait is bounded: after kSpinLimit failed polls the waiter raises PODS_STATUS_TIMEOUT, stops
+// waiting for good and carries on with whatever is in the buffers, still arriving on every barrier
+// it owes, so neither it nor its cluster peers can hang; before the CTA returns the producer waits
+// (again with a limit) for any copy still in flight.
+//
+// The per-row scalar inputs (token, its logit, old/ref log-prob, mask and rollout weight, advantage)
+// are gathered beforehand by a small kernel into one 32-byte record per row, so that the exchange
+// warp fetches them with two independent loads, one row ahead.
 
 #include "grpo_loss_common.cuh"
 
@@ -32,30 +47,51 @@ using namespace pods_loss;
 
 namespace {
 
-constexpr int kClBlock = 256;                 // threads per CTA
-constexpr int kChunkVecs = 512;               // 16-byte vectors per bulk copy (8 KB)
-constexpr int kCtrlBytes = 1024;              // barriers, exchange slots and row scalars ahead of the buffer
-constexpr uint32_t kSpinLimit = 1u << 22;     // polls of one mbarrier before giving up
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kProducerWarp = kConsumerWarps;       // warp 8
+constexpr int kExchangeWarp = kConsumerWarps + 1;   // warp 9
+constexpr int kThreads = kConsumers + 64;
+constexpr int kMaxStages = 3;
+constexpr int kMaxCluster = 8;
+constexpr int kMaxSlots = kMaxCluster * kConsumerWarps;   // (m_w, sum_w) pairs per row
+constexpr int kPieceVecs = 512;               // 16-byte vectors per bulk load (8 KB)
+constexpr int kCtrlBytes = 1408;              // barriers, exchange slots and row scalars ahead of the buffers
+constexpr uint32_t kSpinLimit = 1u << 24;     // polls of one barrier or slot before giving up (a fraction of a second)
+constexpr uint32_t kSuspendNs = 1000;         // upper bound on the time one poll may suspend the thread
 
-struct ClusterCtrl {
-    unsigned long long full;                  // mbarrier of the row's load
-    unsigned long long xkey[2];               // this CTA's arg-max key, read by the peers (slot = row parity:
-    double xsum[2];                           // this CTA's partial sum      a slow peer may still be reading the
-                                              //                             previous row's pair)
-    unsigned long long red_k[kClBlock / 32];
-    double red_d[kClBlock / 32];
-    RowInputs in;                             // scalar inputs of the current row
-    float x_tok;
-    int token;
-    float coef, target;
-    int write_mode;
+struct Pair {
+    uint32_t key;                             // ordered bf16 slice maximum in the upper half
+    float sum;                                // sum of 2^(x log2e - ref_w) over the slice, one maximum left out
 };
-static_assert(sizeof(ClusterCtrl) <= kCtrlBytes, "control block too large");
+
+struct RowPublish {                           // what back(i) needs, per row parity
+    float coef[kConsumerWarps];
+    float target;
+    int write_mode;
+    int token;
+    int pad;
+};
+
+struct Ctrl {
+    unsigned long long full[kMaxStages];      // producer -> consumers: the stage's segment has landed
+    unsigned long long done[kMaxStages];      // consumers -> producer: the stage has been read for the last time
+    unsigned long long sumdone[2];            // consumers -> exchange: the CTA's pairs of the row are in `part`
+    unsigned long long ready[2];              // exchange -> consumers: `pub` of the row is valid
+    Pair part[2][kConsumerWarps];
+    unsigned long long xslot[2][kMaxSlots];   // slot [parity][8 rank + warp] is written by CTA `rank` of the cluster:
+                                              // (sum_w bits) << 32 | (ordered bf16 m_w) << 16 | tag of the row
+    RowPublish pub[2];
+};
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
@@ -64,12 +100,12 @@ __device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
-// Bounded wait; returns false if the barrier did not complete within `limit` polls.
+// Bounded waits; return false if the barrier did not complete within `limit` polls.
 __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, uint32_t limit) {
     for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
@@ -80,31 +116,39 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                 ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// The same barrier for warps that neither published nor will read anything remote: no fences.
-__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait_only() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ unsigned long long ld_peer_u64(const void* local, uint32_t rank) {
+__device__ __forceinline__ uint32_t peer_address(const void* local, uint32_t rank) {
     uint32_t ra;
-    unsigned long long v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(smem_u32(local)), "r"(rank));
-    asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(ra) : "memory");
+    return ra;
+}
+// One 64-bit store into a slot of a peer's shared memory.  The word carries its own row tag, so the
+// reader needs no barrier and the writer no fence: the reader polls the slot until the tag is the
+// row's (an aligned 64-bit store is seen whole or not at all).
+__device__ __forceinline__ void push_word(uint32_t peer_slot, unsigned long long v) {
+    asm volatile("st.relaxed.cluster.shared::cluster.b64 [%0], %1;" ::"r"(peer_slot), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long poll_word(const unsigned long long* slot) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.cluster.shared::cta.b64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
     return v;
+}
+
+// bf16 value (as fp32, -0 already folded into +0) -> 16-bit key whose unsigned order is the order of the values.
+__device__ __forceinline__ uint32_t ordered16(float v) {
+    const uint32_t u = __float_as_uint(v) >> 16;
+    return (u & 0x8000u) ? (~u & 0xffffu) : (u | 0x8000u);
+}
+__device__ __forceinline__ float from_ordered16(uint32_t o) {
+    const uint32_t u = (o & 0x8000u) ? (o & 0x7fffu) : (~o & 0xffffu);
+    return __uint_as_float(u << 16);
 }
 
 // e = 2^(x log2e - ref) for the eight values of a vector: returns their sum, leaves bf16(e) in q.
@@ -142,13 +186,45 @@ __device__ __forceinline__ uint32_t scale_bf16x2(uint32_t e, uint32_t c_hi, uint
     asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o) : "r"(e), "r"(c_hi), "r"(t));
     return o;
 }
+__device__ __forceinline__ void scale_vec(uint4& q, uint32_t c_hi, uint32_t c_lo) {
+    q.x = scale_bf16x2(q.x, c_hi, c_lo);
+    q.y = scale_bf16x2(q.y, c_hi, c_lo);
+    q.z = scale_bf16x2(q.z, c_hi, c_lo);
+    q.w = scale_bf16x2(q.w, c_hi, c_lo);
+}
 
-template <int CL>
-__global__ void __launch_bounds__(kClBlock)
-grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs) {
+__device__ __forceinline__ void max_vec(uint32_t (&pm)[4], const uint4& q) {
+    pm[0] = max_bf16x2(pm[0], q.x);
+    pm[1] = max_bf16x2(pm[1], q.y);
+    pm[2] = max_bf16x2(pm[2], q.z);
+    pm[3] = max_bf16x2(pm[3], q.w);
+}
+
+// One record per row with everything the objective needs besides the logits.
+__global__ void __launch_bounds__(256)
+grpo_row_prep_kernel(const RowArgs a, RowPrep* __restrict__ prep) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= a.T) return;
+    int tok = a.tokens[t];
+    if (tok < 0 || tok >= a.V) { tok = 0; pods_raise(a.status, PODS_STATUS_TOKEN_RANGE); }
+    const RowInputs in = load_row_inputs(a, t);
+    RowPrep r;
+    r.w = in.w;
+    r.adv = (float)in.adv;
+    r.x_tok = __uint_as_float((uint32_t)a.logits[t * a.ldl + tok] << 16);
+    r.old_logp = (float)in.old_logp;
+    r.ref_logp = (float)in.ref_logp;
+    r.token = tok;
+    r.pad = 0;
+    prep[t] = r;
+}
+
+template <int CL, int IT>
+__global__ void __launch_bounds__(kThreads, 2)
+grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages) {
     extern __shared__ __align__(128) unsigned char smem[];
-    ClusterCtrl& c = *reinterpret_cast<ClusterCtrl*>(smem);
-    uint4* buf = reinterpret_cast<uint4*>(smem + kCtrlBytes);
+    Ctrl& c = *reinterpret_cast<Ctrl*>(smem);
+    uint4* const bufs = reinterpret_cast<uint4*>(smem + kCtrlBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_rank();
@@ -156,198 +232,317 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs) {
     const int nvec = a.V / 8;
     const int seg0 = (int)rank * seg_vecs;                                   // first vector of my segment
     const int cnt = max(0, min(seg_vecs, nvec - seg0));                      // vectors in my segment
+    const int64_t n_rows = cluster_id < a.T ? (a.T - cluster_id + n_clusters - 1) / n_clusters : 0;
+    const bool has_ref = a.ref_logp != nullptr && a.beta != 0.0f;
 
+    if (tid < 2 * kMaxSlots) (&c.xslot[0][0])[tid] = 0ull;         // tag 0 is no row's tag
     if (tid == 0) {
-        mbar_init(&c.full, 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(&c.full[s], 1);                  // the copy issuer, with the byte count
+            mbar_init(&c.done[s], kConsumerWarps);
+        }
+        for (int p = 0; p < 2; ++p) {
+            mbar_init(&c.sumdone[p], kConsumerWarps);
+            mbar_init(&c.ready[p], kConsumerWarps);    // the eight lanes that publish a coefficient each
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    cluster_sync();                                    // every slot of the cluster is cleared before anyone writes to it
 
-    uint32_t parity = 0;
     bool timed_out = false;
-    for (int64_t t = cluster_id; t < a.T; t += n_clusters, parity ^= 1u) {
-        const uint16_t* row = a.logits + t * a.ldl;
-        uint16_t* drow = a.dlogits + t * a.ldd;
 
-        // ---- load ------------------------------------------------------------------------------
-        if (tid == 0) {
-            bulk_wait_read();                      // the previous row's store has finished reading buf
-            mbar_expect_tx(&c.full, (uint32_t)cnt * 16u);
-            for (int v0 = 0; v0 < cnt; v0 += kChunkVecs)
-                bulk_load(buf + v0, reinterpret_cast<const uint4*>(row) + seg0 + v0,
-                          (uint32_t)min(kChunkVecs, cnt - v0) * 16u, &c.full);
-        } else if (tid == 32) {
-            int tok = a.tokens[t];
-            if (tok < 0 || tok >= a.V) { tok = 0; if (rank == 0) pods_raise(a.status, PODS_STATUS_TOKEN_RANGE); }
-            c.token = tok;
-            c.x_tok = __uint_as_float((uint32_t)row[tok] << 16);   // before any peer stores this row in place
-            c.in = load_row_inputs(a, t);
-        }
-        // after one timeout the CTA stops waiting for good: it fails fast instead of stalling per row
-        if (!mbar_wait(&c.full, parity, timed_out ? 1u : kSpinLimit)) timed_out = true;
-
-        // ---- max of my segment -------------------------------------------------------------------
-        float m_t = -INFINITY;
-        int pos_t = 0x7fffffff;
-#pragma unroll 4
-        for (int j = tid; j < cnt; j += kClBlock) {
-            const float vm = vec_max(buf[j]);
-            const bool up = vm > m_t;
-            m_t = up ? vm : m_t;
-            pos_t = up ? j : pos_t;
-        }
-        unsigned long long key = argmax_key(m_t, pos_t);
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(PODS_FULL_MASK, key, d);
-            key = o > key ? o : key;
-        }
-        if (lane == 0) c.red_k[warp] = key;
-        __syncthreads();
-        unsigned long long seg_key = c.red_k[0];
-#pragma unroll
-        for (int w = 1; w < kClBlock / 32; ++w) seg_key = c.red_k[w] > seg_key ? c.red_k[w] : seg_key;
-        const float m_r = argmax_key_value(seg_key);
-        const int excl = argmax_key_pos(seg_key);                              // local vector of the left-out instance
-        const float ref_r = m_r * kLog2e;
-
-        // ---- sum, bf16(e) written back in place --------------------------------------------------
-        float s_t = 0.0f;
-        if (excl < cnt && (excl % kClBlock) == tid) s_t = exp_sum_excluding(buf[excl], ref_r, m_r);
-#pragma unroll 2
-        for (int j = tid; j < cnt; j += kClBlock) {
-            uint4 q = buf[j];
-            const float sum = exp_vec_inplace(q, ref_r);
-            s_t += (j == excl) ? 0.0f : sum;
-            buf[j] = q;
-        }
-        double sd = (double)s_t;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) sd += __shfl_xor_sync(PODS_FULL_MASK, sd, d);
-        if (lane == 0) c.red_d[warp] = sd;
-        __syncthreads();
-
-        // ---- share: one cluster barrier, then the scalar terms on warp 0 -----------------------
-        if (warp == 0) {
-            if (lane == 0) {
-                double s = 0.0;
-#pragma unroll
-                for (int w = 0; w < kClBlock / 32; ++w) s += c.red_d[w];
-                c.xkey[parity] = seg_key;
-                c.xsum[parity] = s;
+    if (warp == kProducerWarp) {
+        // =================================== producer (one thread) ===================================
+        if (lane == 0) {
+            // issue(i, s): the loads of row i into stage s
+            auto issue = [&](int64_t i, int s) {
+                const int64_t t = cluster_id + i * n_clusters;
+                const uint4* src = reinterpret_cast<const uint4*>(a.logits + t * a.ldl) + seg0;
+                if (cnt > 0) {
+                    mbar_expect_tx(&c.full[s], (uint32_t)cnt * 16u);
+                    uint4* dst = bufs + (size_t)s * seg_vecs;
+                    for (int v0 = 0; v0 < cnt; v0 += kPieceVecs)
+                        bulk_load(dst + v0, src + v0, (uint32_t)min(kPieceVecs, cnt - v0) * 16u, &c.full[s]);
+                } else {
+                    mbar_arrive(&c.full[s]);
+                }
+            };
+            const int64_t ahead = n_rows < n_stages ? n_rows : n_stages;
+            for (int64_t i = 0; i < ahead; ++i) issue(i, (int)i);
+            int s = 0;
+            uint32_t parity = 0;
+            for (int64_t i = 0; i + n_stages < n_rows; ++i) {
+                if (!mbar_wait(&c.done[s], parity, timed_out ? 1u : kSpinLimit)) timed_out = true;
+                issue(i + n_stages, s);
+                if (++s == n_stages) { s = 0; parity ^= 1u; }
             }
-            __syncwarp();
-            cluster_sync();                                                    // release my pair, acquire the peers'
-            // lane r < CL holds the pair of rank r
-            unsigned long long k_r = 0ull;
-            double s_r = 0.0;
-            if (lane < CL) {
-                k_r = ld_peer_u64(&c.xkey[parity], lane);
-                s_r = __longlong_as_double((long long)ld_peer_u64(&c.xsum[parity], lane));
+            // a consumer may have given up on a load that is still in flight: every load has to have landed
+            // before the CTA ends (the waits return at once when nothing went wrong)
+            for (int st = 0; st < n_stages; ++st) {
+                const int64_t uses = n_rows > st ? (n_rows - st + n_stages - 1) / n_stages : 0;
+                if (uses > 0 && !mbar_wait(&c.full[st], (uint32_t)((uses - 1) & 1), kSpinLimit)) timed_out = true;
             }
-            // the row maximum; among equal maxima the lowest rank's instance is the one left out
-            const float mr = argmax_key_value(k_r);
-            unsigned long long best = lane < CL ? (k_r & 0xffffffff00000000ull) | (uint32_t)(0xffu - lane) : 0ull;
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const unsigned long long o = __shfl_xor_sync(PODS_FULL_MASK, best, d);
-                best = o > best ? o : best;
+        }
+        __syncwarp();
+    } else if (warp == kExchangeWarp) {
+        // =================================== exchange warp ===================================
+        const int n_slots = CL * kConsumerWarps;
+        const uint4* prep4 = reinterpret_cast<const uint4*>(a.prep);
+        // the row's scalar inputs, fetched one row ahead (every lane reads the same two vectors)
+        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+        if (n_rows > 0) { nx0 = prep4[2 * cluster_id]; nx1 = prep4[2 * cluster_id + 1]; }
+        for (int64_t i = 0; i < n_rows; ++i) {
+            const uint32_t xp = (uint32_t)(i & 1), xparity = (uint32_t)((i >> 1) & 1);
+            const int64_t t = cluster_id + i * n_clusters;
+            RowPrep in;
+            in.w = __hiloint2double((int)nx0.y, (int)nx0.x);
+            in.adv = __uint_as_float(nx0.z);
+            in.x_tok = __uint_as_float(nx0.w);
+            in.old_logp = __uint_as_float(nx1.x);
+            in.ref_logp = __uint_as_float(nx1.y);
+            in.token = (int)nx1.z;
+            if (i + 1 < n_rows) { nx0 = prep4[2 * (t + n_clusters)]; nx1 = prep4[2 * (t + n_clusters) + 1]; }
+            if (!mbar_wait(&c.sumdone[xp], xparity, timed_out ? 1u : kSpinLimit)) timed_out = true;
+            // lane l pushes pair (l % 8) of this CTA to peers l / 8 and l / 8 + 4
+            const unsigned long long tag = (unsigned long long)((i + 1) & 0xffff);
+            {
+                const int w = lane & 7;
+                const Pair mine = c.part[xp][w];
+                const unsigned long long word = ((unsigned long long)__float_as_uint(mine.sum) << 32) |
+                                                (unsigned long long)(mine.key & 0xffff0000u) | tag;
+                for (uint32_t peer = (uint32_t)lane >> 3; peer < (uint32_t)CL; peer += 4)
+                    push_word(peer_address(&c.xslot[xp][rank * kConsumerWarps + w], peer), word);
             }
-            const float mx = argmax_key_value(best);
-            const int owner = 0xff - (int)(best & 0xffu);
-            // sum_r is relative to ref_r: bring it to the row maximum; every segment but the owner's
-            // gets back the instance of its own maximum that it left out
-            double scale_r = 0.0, contrib = 0.0;
-            if (lane < CL && mr != -INFINITY) {
-                scale_r = exp((double)(mr - mx));
-                const double true_r = s_r * ref_correction(mr, mr * kLog2e);
-                contrib = (lane == owner) ? true_r : (true_r + 1.0) * scale_r;
+            // lane l collects slots l and l + 32: polls until both carry the row's tag
+            unsigned long long w0 = tag, w1 = tag;
+            {
+                const uint32_t limit = timed_out ? 1u : kSpinLimit;
+                uint32_t it = 0;
+                for (;;) {
+                    if (lane < n_slots) w0 = poll_word(&c.xslot[xp][lane]);
+                    if (lane + 32 < n_slots) w1 = poll_word(&c.xslot[xp][lane + 32]);
+                    const bool ok = (w0 & 0xffffull) == tag && (w1 & 0xffffull) == tag;
+                    if (__all_sync(PODS_FULL_MASK, ok)) break;
+                    if (++it >= limit) { timed_out = true; break; }
+                }
+            }
+            // lane l holds slots l and l + 32
+            Pair p0, p1;
+            p0.key = (uint32_t)w0 & 0xffff0000u;
+            p0.sum = __uint_as_float((uint32_t)(w0 >> 32));
+            p1.key = (uint32_t)w1 & 0xffff0000u;
+            p1.sum = __uint_as_float((uint32_t)(w1 >> 32));
+            // the row maximum; among equal maxima the lowest slot's instance is the one left out of the sums
+            const uint32_t cand0 = lane < n_slots ? ((p0.key & 0xffff0000u) | (uint32_t)(0xffff - lane)) : 0u;
+            const uint32_t cand1 = lane + 32 < n_slots ? ((p1.key & 0xffff0000u) | (uint32_t)(0xffff - lane - 32)) : 0u;
+            const uint32_t best = __reduce_max_sync(PODS_FULL_MASK, max(cand0, cand1));
+            const float mx = from_ordered16(best >> 16);
+            const int owner_slot = 0xffff - (int)(best & 0xffffu);
+            // the exponentials of the scalar terms need only the maximum: three lanes, three calls at once
+            const double xr = (double)in.x_tok - (double)mx;                   // <= 0
+            // lane 0: rho Z, lane 1: e^d / Z, lane 2: p Z (one call, a different argument per lane)
+            const double part = exp(lane == 0 ? xr - (double)in.old_logp : (lane == 1 ? (double)in.ref_logp - xr : xr));
+            // sum_w is relative to ref_w: bring it to the row maximum; every slice but the owner's gets back
+            // the instance of its own maximum that it left out
+            const float m0 = from_ordered16(p0.key >> 16), m1 = from_ordered16(p1.key >> 16);
+            float scale0 = 0.0f, scale1 = 0.0f;
+            double contrib = 0.0;
+            if (lane < n_slots && m0 != -INFINITY) {
+                scale0 = ex2_approx((m0 - mx) * kLog2e);
+                const double tr = (double)p0.sum * ref_correction(m0, m0 * kLog2e);
+                contrib += (lane == owner_slot) ? tr : (tr + 1.0) * (double)scale0;
+            }
+            if (lane + 32 < n_slots && m1 != -INFINITY) {
+                scale1 = ex2_approx((m1 - mx) * kLog2e);
+                const double tr = (double)p1.sum * ref_correction(m1, m1 * kLog2e);
+                contrib += (lane + 32 == owner_slot) ? tr : (tr + 1.0) * (double)scale1;
             }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) contrib += __shfl_xor_sync(PODS_FULL_MASK, contrib, d);
             const double zp = contrib;                                         // Z - 1
-            const double my_scale = __shfl_sync(PODS_FULL_MASK, scale_r, (int)rank);
-            // scalar terms: the transcendental calls on three lanes at once
-            const RowInputs in = c.in;
-            const float x_tok = c.x_tok;
-            const double logp = ((double)x_tok - (double)mx) - log1p(zp);
-            double part = 0.0;
-            if (lane == 0) part = exp(logp - in.old_logp);                     // rho
-            else if (lane == 1) part = in.has_ref ? exp(in.ref_logp - logp) : 1.0;    // e^d
-            else if (lane == 2) part = (x_tok == mx) ? zp / (1.0 + zp) : -expm1(logp);   // 1 - p
-            const double rho = __shfl_sync(PODS_FULL_MASK, part, 0);
-            const double ed = __shfl_sync(PODS_FULL_MASK, part, 1);
-            const double one_minus_p = __shfl_sync(PODS_FULL_MASK, part, 2);
-            if (lane == 0) {
-                const double eps = (double)a.eps, beta = (double)a.beta;
-                const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
-                const double s1 = rho * in.adv, s2 = clipped * in.adv;
-                double loss = -(s1 < s2 ? s1 : s2);
-                double dl = (s1 <= s2) ? -in.adv * rho : 0.0;
-                if (in.has_ref) {
-                    const double d = in.ref_logp - logp;
+            const double Z = 1.0 + zp;
+            const double inv_z = 1.0 / Z;
+            // the factors of this CTA's own slices: slot rank * 8 + w sits in lane (rank * 8 + w) % 32
+            const int my_slot = (int)rank * kConsumerWarps + (lane & 7);
+            const float sc_lo = __shfl_sync(PODS_FULL_MASK, scale0, my_slot & 31);
+            const float sc_hi = __shfl_sync(PODS_FULL_MASK, scale1, my_slot & 31);
+            const float mw_lo = __shfl_sync(PODS_FULL_MASK, m0, my_slot & 31);
+            const float mw_hi = __shfl_sync(PODS_FULL_MASK, m1, my_slot & 31);
+            const float my_scale = my_slot < 32 ? sc_lo : sc_hi;
+            const float my_m = my_slot < 32 ? mw_lo : mw_hi;
+            const double adv = (double)in.adv;
+            const double rho = __shfl_sync(PODS_FULL_MASK, part, 0) * inv_z;
+            const double ed = has_ref ? __shfl_sync(PODS_FULL_MASK, part, 1) * Z : 1.0;
+            const double pz = __shfl_sync(PODS_FULL_MASK, part, 2);
+            // 1 - p: exact route when the target holds the maximum (p may be close to 1), plain otherwise (p < 1/2)
+            const double one_minus_p = (in.x_tok == mx) ? zp * inv_z : 1.0 - pz * inv_z;
+            const double eps = (double)a.eps, beta = (double)a.beta;
+            const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
+            const double t1 = rho * adv, t2 = clipped * adv;
+            double dl = (t1 <= t2) ? -adv * rho : 0.0;
+            if (has_ref) dl += beta * (1.0 - ed);
+            const double g = (in.w != 0.0) ? (double)a.grad_scale * in.w * dl : 0.0;
+            if (lane < kConsumerWarps) {
+                // e^(x - M) = e_stored * 2^(ref_w - m_w log2e) * e^(m_w - M)
+                c.pub[xp].coef[lane] = (float)(-g * inv_z * ref_correction(my_m, my_m * kLog2e) * (double)my_scale);
+                if (lane == 0) {
+                    c.pub[xp].target = (float)(g * one_minus_p);
+                    c.pub[xp].write_mode = (g != 0.0) ? 1 : 0;
+                    c.pub[xp].token = in.token;
+                }
+                mbar_arrive(&c.ready[xp]);
+            }
+            // ---- nobody waits for these: the log-prob and the row's loss term --------------------------
+            if (rank == 0 && lane == 0) {
+                const double logp = xr - log1p(zp);
+                double loss = -(t1 < t2 ? t1 : t2);
+                if (has_ref) {
+                    const double d = (double)in.ref_logp - logp;
                     loss += beta * (ed - d - 1.0);
-                    dl += beta * (1.0 - ed);
                 }
-                const double g = (in.w != 0.0) ? (double)a.grad_scale * in.w * dl : 0.0;
-                if (rank == 0) {
-                    a.logp[t] = (float)logp;
-                    a.row_loss[t] = (in.w != 0.0) ? in.w * loss : 0.0;   // a masked row adds nothing, whatever its inputs
+                a.logp[t] = (float)logp;
+                a.row_loss[t] = (in.w != 0.0) ? in.w * loss : 0.0;   // a masked row adds nothing, whatever its inputs
+            }
+            __syncwarp();
+        }
+    } else {
+        // =================================== consumer warps ===================================
+        const int per_warp = (cnt + kConsumerWarps - 1) / kConsumerWarps;
+        const int lo = min(cnt, warp * per_warp), hi = min(cnt, lo + per_warp);    // my slice of the segment
+        const uint4 kNegInf4 = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+
+        // back(i): the gradient of row i over my slice, once the exchange warp has published its factors
+        auto back = [&](int64_t i, int s) {
+            const uint32_t xp = (uint32_t)(i & 1);
+            const uint4* const buf = bufs + (size_t)s * seg_vecs;
+            const int64_t t = cluster_id + i * n_clusters;
+            uint4* const out = reinterpret_cast<uint4*>(a.dlogits + t * a.ldd) + seg0;
+            if (!mbar_wait(&c.ready[xp], (uint32_t)((i >> 1) & 1), timed_out ? 1u : kSpinLimit)) timed_out = true;
+            if (c.pub[xp].write_mode == 0) {
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int k = 0; k < IT; ++k) {
+                    const int j = lo + lane + 32 * k;
+                    if (j < hi) __stcs(out + j, z);
                 }
-                // e^(x - M) = e_stored * 2^(ref_r - m_r log2e) * e^(m_r - M)
-                c.coef = (float)(-g / (1.0 + zp) * ref_correction(m_r, ref_r) * my_scale);
-                c.target = (float)(g * one_minus_p);
-                c.write_mode = (g != 0.0) ? 1 : 0;
+            } else {
+                const float coef = c.pub[xp].coef[warp];
+                const uint16_t hi16 = to_bf16_bits(coef);
+                const uint16_t lo16 = to_bf16_bits(coef - __uint_as_float((uint32_t)hi16 << 16));
+                const uint32_t c_hi = (uint32_t)hi16 * 0x10001u, c_lo = (uint32_t)lo16 * 0x10001u;
+                const int token = c.pub[xp].token;
+                const int tok_vec = (token >> 3) - seg0;                        // the vector with the target entry, if it is mine
+                const uint16_t target_bits = to_bf16_bits(c.pub[xp].target);
+                uint4 q[IT];
+#pragma unroll
+                for (int k = 0; k < IT; ++k) {
+                    const int j = lo + lane + 32 * k;
+                    q[k] = j < hi ? buf[j] : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < IT; ++k) {
+                    const int j = lo + lane + 32 * k;
+                    scale_vec(q[k], c_hi, c_lo);
+                    if (j == tok_vec) patch_bf16(q[k], token & 7, target_bits);
+                    if (j < hi) __stcs(out + j, q[k]);
+                }
             }
-        } else {
-            cluster_arrive_relaxed();
-        }
-        __syncthreads();
-        if (warp != 0) cluster_wait_only();        // completes at once: warp 0 is already past it
+            __syncwarp();                              // every lane has its values: the stage may be loaded again
+            if (lane == 0) mbar_arrive(&c.done[s]);
+        };
 
-        // ---- grad, in place ------------------------------------------------------------------------
-        if (c.write_mode == 0) {
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            for (int j = tid; j < cnt; j += kClBlock) buf[j] = z;
-        } else {
-            const float coef = c.coef;
-            const uint16_t hi16 = to_bf16_bits(coef);
-            const uint16_t lo16 = to_bf16_bits(coef - __uint_as_float((uint32_t)hi16 << 16));
-            const uint32_t c_hi = (uint32_t)hi16 * 0x10001u, c_lo = (uint32_t)lo16 * 0x10001u;
-#pragma unroll 4
-            for (int j = tid; j < cnt; j += kClBlock) {
-                uint4 q = buf[j];
-                q.x = scale_bf16x2(q.x, c_hi, c_lo);
-                q.y = scale_bf16x2(q.y, c_hi, c_lo);
-                q.z = scale_bf16x2(q.z, c_hi, c_lo);
-                q.w = scale_bf16x2(q.w, c_hi, c_lo);
-                buf[j] = q;
+        int s = 0, s_prev = 0;
+        uint32_t parity = 0;
+        for (int64_t i = 0; i < n_rows; ++i) {
+            const uint32_t xp = (uint32_t)(i & 1);
+            uint4* const buf = bufs + (size_t)s * seg_vecs;
+
+            if (!mbar_wait(&c.full[s], parity, timed_out ? 1u : kSpinLimit)) timed_out = true;
+
+            // ---- my slice into registers; its maximum ------------------------------------------
+            uint4 q[IT];
+#pragma unroll
+            for (int k = 0; k < IT; ++k) {
+                const int j = lo + lane + 32 * k;
+                q[k] = j < hi ? buf[j] : kNegInf4;
             }
-            const int tok_vec = (c.token >> 3) - seg0;                         // the target entry, if it is mine:
-            if (tok_vec >= 0 && tok_vec < cnt && (tok_vec % kClBlock) == tid)  // rewritten by the thread that wrote it
-                reinterpret_cast<uint16_t*>(buf)[tok_vec * 8 + (c.token & 7)] = to_bf16_bits(c.target);
-        }
-        fence_proxy_async();                       // my shared-memory writes, before the bulk copy reads them
-        __syncthreads();
+            uint32_t pm[4] = {kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair};
+#pragma unroll
+            for (int k = 0; k < IT; ++k) max_vec(pm, q[k]);
+            const uint32_t pmax = max_bf16x2(max_bf16x2(pm[0], pm[1]), max_bf16x2(pm[2], pm[3]));
+            const float m_t = fmaxf(bf16_lo(pmax), bf16_hi(pmax)) + 0.0f;             // -0 -> +0
+            const uint32_t key_w = __reduce_max_sync(PODS_FULL_MASK, (ordered16(m_t) << 16) | (uint32_t)(31 - lane));
+            const float m_w = from_ordered16(key_w >> 16);
+            const int owner = 31 - (int)(key_w & 0xffffu);               // lowest lane that holds an instance of m_w
+            const float ref_w = m_w * kLog2e;
+            // which of the owner's vectors holds it: the first k with that maximum (-1 on every other lane)
+            int excl = -1;
+            {
+                // lane k looks at the owner's k-th vector (still unmodified in shared memory)
+                const int j = lo + owner + 32 * lane;
+                const bool hit = lane < IT && j < hi && vec_max(buf[j]) == m_w;
+                const uint32_t hits = __ballot_sync(PODS_FULL_MASK, hit);
+                if (lane == owner && hits != 0u) excl = __ffs(hits) - 1;
+            }
 
-        // ---- store ---------------------------------------------------------------------------------
-        if (tid == 0 && cnt > 0)
-            bulk_store(reinterpret_cast<uint4*>(drow) + seg0, buf, (uint32_t)cnt * 16u);
+            // ---- sum, bf16(e) written back in place ----------------------------------------------
+            float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < IT; ++k) {
+                const int j = lo + lane + 32 * k;
+                const float part = (k == excl) ? exp_sum_excluding(q[k], ref_w, m_w) : 0.0f;
+                const float sum = exp_vec_inplace(q[k], ref_w);
+                if (k & 1) s1 += (k == excl) ? part : sum; else s0 += (k == excl) ? part : sum;
+                if (j < hi) buf[j] = q[k];
+            }
+            float sw = s0 + s1;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) sw += __shfl_xor_sync(PODS_FULL_MASK, sw, d);
+            if (lane == 0) {
+                Pair mine;
+                mine.key = key_w & 0xffff0000u;
+                mine.sum = sw;
+                c.part[xp][warp] = mine;
+                mbar_arrive(&c.sumdone[xp]);
+            }
+
+            if (i > 0) back(i - 1, s_prev);
+            s_prev = s;
+            if (++s == n_stages) { s = 0; parity ^= 1u; }
+        }
+        if (n_rows > 0) back(n_rows - 1, s_prev);
     }
-    if (tid == 0) bulk_wait_all();
     if (timed_out && lane == 0) pods_raise(a.status, PODS_STATUS_TIMEOUT);
-    cluster_sync();                                // no CTA leaves while a peer may still read its exchange slots
+    cluster_sync();                                    // no CTA leaves while a peer may still write its exchange slots
 }
 
-template <int CL>
-int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
-    *launched = false;
-    const int nvec = a.V / 8;
-    int seg_vecs = (nvec + CL - 1) / CL;
-    const size_t smem = (size_t)kCtrlBytes + (size_t)seg_vecs * 16;
-    if (smem > 227 * 1024 || (size_t)seg_vecs * 16 >= (1u << 20)) return PODS_OK;     // does not fit: caller falls back
-    auto kernel = grpo_loss_cluster_kernel<CL>;
-    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+struct ClusterPlan {
+    int seg_vecs, n_stages;
+    size_t smem;
+};
+
+// Ring depth and residency for a row of nvec vectors over `cl` CTAs: three stages (one row being
+// loaded, one in front(), one waiting for back()) and as many CTAs per SM as then fit; two stages
+// when three do not fit at all.
+bool plan_cluster(int nvec, int cl, ClusterPlan* p) {
+    const size_t limit = 232448;
+    p->seg_vecs = (nvec + cl - 1) / cl;
+    const size_t seg_bytes = (size_t)p->seg_vecs * 16;
+    if (seg_bytes >= (1u << 20)) return false;
+    for (int stages = kMaxStages; stages >= 2; --stages) {
+        p->n_stages = stages;
+        p->smem = kCtrlBytes + (size_t)stages * seg_bytes;
+        if (p->smem <= limit) return true;
+    }
+    return false;
+}
+
+template <int CL, int IT>
+int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t stream, bool* launched) {
+    ClusterPlan plan = plan_in;
+    auto kernel = grpo_loss_cluster_kernel<CL, IT>;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -355,8 +550,8 @@ int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.gridDim = dim3(CL, 1, 1);
-    cfg.blockDim = dim3(kClBlock, 1, 1);
-    cfg.dynamicSmemBytes = smem;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
@@ -365,9 +560,28 @@ int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     if (max_clusters < 1) return PODS_OK;
     const int64_t n_clusters = a.T < max_clusters ? a.T : max_clusters;
     cfg.gridDim = dim3((unsigned)(n_clusters * CL), 1, 1);
-    PODS_RETURN_IF_CUDA_ERROR(cudaLaunchKernelEx(&cfg, kernel, a, seg_vecs));
+    grpo_row_prep_kernel<<<(unsigned)((a.T + 255) / 256), 256, 0, stream>>>(a, a.prep);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    PODS_RETURN_IF_CUDA_ERROR(cudaLaunchKernelEx(&cfg, kernel, a, plan.seg_vecs, plan.n_stages));
     *launched = true;
     return PODS_OK;
+}
+
+// IT = vectors per lane of a consumer warp's slice, rounded up to the next instantiated depth.
+template <int CL>
+int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
+    *launched = false;
+    ClusterPlan plan;
+    if (!plan_cluster(a.V / 8, CL, &plan)) return PODS_OK;                 // does not fit: caller falls back
+    const int per_warp = (plan.seg_vecs + kConsumerWarps - 1) / kConsumerWarps;
+    const int it = (per_warp + 31) / 32;
+    if (it <= 2) return launch_cluster_it<CL, 2>(a, plan, stream, launched);
+    if (it <= 4) return launch_cluster_it<CL, 4>(a, plan, stream, launched);
+    if (it <= 6) return launch_cluster_it<CL, 6>(a, plan, stream, launched);
+    if (it <= 8) return launch_cluster_it<CL, 8>(a, plan, stream, launched);
+    if (it <= 10) return launch_cluster_it<CL, 10>(a, plan, stream, launched);
+    if (it <= 12) return launch_cluster_it<CL, 12>(a, plan, stream, launched);
+    return PODS_OK;                                                        // rows too long for the register-held slices
 }
 
 }  // namespace

@@ -72,6 +72,16 @@ __device__ __forceinline__ int argmax_key_pos(unsigned long long k) {
     return 0x7fffffff - (int)(uint32_t)(k & 0xffffffffu);
 }
 
+// Everything the objective needs for one row besides the logits, gathered by the cluster path's
+// preparation kernel: 32 bytes, read as two 16-byte vectors.
+struct __align__(16) RowPrep {
+    double w;            // mask_t / (M |o_i|)
+    float adv, x_tok;    // advantage of the row's rollout; the target's logit
+    float old_logp, ref_logp;
+    int token;
+    int pad;
+};
+
 struct RowArgs {
     const uint16_t* logits;
     int64_t ldl;
@@ -91,6 +101,7 @@ struct RowArgs {
     uint16_t* dlogits;
     int64_t ldd;
     double* row_loss;      // workspace [T]: mask_t w_i loss_t
+    RowPrep* prep;         // workspace [T]: the rows' scalar inputs (cluster path)
     uint32_t* status;
     int vec_ok;            // 16-byte aligned rows: 128-bit path
 };
