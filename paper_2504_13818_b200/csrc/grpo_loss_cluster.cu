@@ -19,9 +19,10 @@
 //                        when one logit dominates), bf16(e) written back to shared memory in place;
 //                        (m_w, sum_w) is handed to the exchange warp;
 //       back(i-1) grad   bf16(coef_w * e) by packed bf16 multiply-adds with coef_w split into two
-//                        bf16 terms (coef_w folds in 2^(ref_w - M log2e)), the target entry replaced
-//                        by g (1 - p), stored straight to global memory with 128-bit streaming
-//                        stores; the warp then arrives on the stage's `done` barrier.
+//                        bf16 terms (coef_w folds in 2^(ref_w - M log2e)), stored straight to global
+//                        memory with 128-bit streaming stores, the target entry then overwritten
+//                        with g (1 - p) by the lane that stored its vector; the warp then arrives
+//                        on the stage's `done` barrier.
 //             front(i) runs before back(i-1), so the exchange of row i-1 has a whole sweep to finish.
 //             Shared memory sees 8 bytes of traffic per element (2 in, 2 read, 2 written, 2 read).
 //   exchange  for every row: writes the CTA's eight (m_w, sum_w) pairs into the slots it owns in
@@ -444,9 +445,11 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 for (int k = 0; k < IT; ++k) {
                     const int j = lo + lane + 32 * k;
                     scale_vec(q[k], c_hi, c_lo);
-                    if (j == tok_vec) patch_bf16(q[k], token & 7, target_bits);
                     if (j < hi) __stcs(out + j, q[k]);
                 }
+                // the target entry, if it is in my slice: rewritten by the lane that stored its vector
+                if (tok_vec >= lo && tok_vec < hi && ((tok_vec - lo) & 31) == lane)
+                    reinterpret_cast<uint16_t*>(out)[(int64_t)tok_vec * 8 + (token & 7)] = target_bits;
             }
             __syncwarp();                              // every lane has its values: the stage may be loaded again
             if (lane == 0) mbar_arrive(&c.done[s]);
