@@ -303,6 +303,263 @@ pods_select_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, i
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Fast path for the max-variance and max-reward rules: the sort carries 32-bit keys only.
+// ---------------------------------------------------------------------------------------------
+// Algorithm 2 needs the sorted VALUES (for the running sums and the scores of the m+1 splits), but
+// which rollouts are kept follows from two thresholds: the kept set is every reward below v_lo (the
+// value at sorted position m-k-1), the first few in index order of those equal to v_lo, every reward
+// above v_hi (the value at sorted position n-k), and the last few in index order of those equal to
+// v_hi - exactly the set the stable (reward, index) order picks.  So the network sorts bare 32-bit
+// keys (one min and one max per compare-exchange, no payload), in the form whose first step of
+// every merge level mirrors the block (position p against p ^ (k-1)) so that all steps put the
+// minimum at the lower position and no direction has to be selected.  A second sweep over the
+// rewards in original order (kept in registers) then emits indices and advantages.
+
+// key at sorted position p of the group (positions are blocked: lane sl holds sl*E .. sl*E+E-1)
+template <int LANES, int E>
+__device__ __forceinline__ uint32_t key_at(const uint32_t (&key)[E], int p, int sub) {
+    uint32_t mine = key[0];
+#pragma unroll
+    for (int e = 1; e < E; ++e) mine = ((p & (E - 1)) == e) ? key[e] : mine;
+    return __shfl_sync(PODS_FULL_MASK, mine, sub * LANES + ((p / E) & (LANES - 1)));
+}
+
+template <int LANES, int E>
+__global__ void __launch_bounds__(kSelectThreads)
+pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint32_t flags,
+                        int32_t* __restrict__ idx_out, float* __restrict__ adv_out, int32_t* __restrict__ k_out,
+                        uint32_t* status) {
+    constexpr int NPAD = LANES * E;
+    constexpr int GPW = 32 / LANES;                 // groups per warp
+    constexpr uint32_t GROUP_MASK = LANES == 32 ? 0xffffffffu : ((1u << LANES) - 1u);
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / LANES, sl = lane % LANES;
+    double* PL1 = reinterpret_cast<double*>(smem_raw) + (size_t)(warp * GPW + sub) * 4 * (m + 1);   // sum of the j lowest
+    double* PL2 = PL1 + (m + 1);
+    double* SU1 = PL2 + (m + 1);                        // sum of the m-j highest, j = 0..m
+    double* SU2 = SU1 + (m + 1);
+
+    const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
+    for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
+        const int64_t g = base + sub;
+        const bool valid = g < G;
+        const float* r_g = rewards + (valid ? g : 0) * (int64_t)n;
+
+        // ---- 1. load (coalesced: lane sl holds original indices e*LANES + sl) and key -----------
+        float orig[E];
+        uint32_t key[E];
+        bool nonfinite = false;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int i = e * LANES + sl;
+            orig[e] = (i < n && valid) ? r_g[i] : 0.0f;
+            nonfinite |= !(fabsf(orig[e]) <= 3.402823466e38f);
+            key[e] = i < n ? ordered_bits(orig[e]) : 0xffffffffu;     // padding sorts last (with the NaNs, whose key it shares)
+        }
+        if (nonfinite && valid) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
+
+        // ---- 2. bitonic sort of the keys over positions p = sl * E + e ------------------------------
+#pragma unroll
+        for (int k = 2; k <= NPAD; k <<= 1) {
+            // mirror step: p against p ^ (k - 1)
+            if (k <= E) {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const int f = e ^ (k - 1);
+                    if (e < f) {
+                        const uint32_t a = key[e], b = key[f];
+                        key[e] = min(a, b);
+                        key[f] = max(a, b);
+                    }
+                }
+            } else {
+                const int lane_xor = (k - 1) / E;                      // k / E - 1: all lane bits below k / E
+                const bool lower = (sl & (k / (2 * E))) == 0;
+                uint32_t other[E];
+#pragma unroll
+                for (int e = 0; e < E; ++e) other[e] = __shfl_xor_sync(PODS_FULL_MASK, key[E - 1 - e], lane_xor);
+#pragma unroll
+                for (int e = 0; e < E; ++e) key[e] = lower ? min(key[e], other[e]) : max(key[e], other[e]);
+            }
+            // the remaining steps of the level: p against p ^ j, minimum to the lower position
+#pragma unroll
+            for (int j = k >> 2; j > 0; j >>= 1) {
+                if (j >= E) {
+                    const int lane_xor = j / E;
+                    const bool lower = (sl & lane_xor) == 0;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const uint32_t other = __shfl_xor_sync(PODS_FULL_MASK, key[e], lane_xor);
+                        key[e] = lower ? min(key[e], other) : max(key[e], other);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if ((e & j) == 0) {
+                            const uint32_t a = key[e], b = key[e | j];
+                            key[e] = min(a, b);
+                            key[e | j] = max(a, b);
+                        }
+                    }
+                }
+            }
+        }
+
+        // ---- 3. centred rewards and fp64 running sums over the sorted order ------------------------
+        const uint32_t first = __shfl_sync(PODS_FULL_MASK, key[0], sub * LANES);
+        const double centre = (double)from_ordered_bits(first);              // the group minimum
+        int kstar = rule == PODS_RULE_MAXREWARD ? m : 0;                      // m == n: every split is the whole group
+        double k1 = 0.0, k2 = 0.0;                                            // sums of x and x^2 over the kept subset
+        double f1 = 0.0, f2 = 0.0;                                            // ... and over the full group
+        {
+            double x[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int p = sl * E + e;
+                x[e] = p < n ? (double)from_ordered_bits(key[e]) - centre : 0.0;
+            }
+            double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) { s1 += x[e]; s2 += x[e] * x[e]; }
+            double i1 = s1, i2 = s2;                         // inclusive scan over the lanes below
+            double j1 = s1, j2 = s2;                         // inclusive scan over the lanes above
+#pragma unroll
+            for (int d = 1; d < LANES; d <<= 1) {
+                const double t1 = __shfl_up_sync(PODS_FULL_MASK, i1, d, LANES);
+                const double t2 = __shfl_up_sync(PODS_FULL_MASK, i2, d, LANES);
+                const double u1 = __shfl_down_sync(PODS_FULL_MASK, j1, d, LANES);
+                const double u2 = __shfl_down_sync(PODS_FULL_MASK, j2, d, LANES);
+                if (sl >= d) { i1 += t1; i2 += t2; }
+                if (sl + d < LANES) { j1 += u1; j2 += u2; }
+            }
+            f1 = __shfl_sync(PODS_FULL_MASK, i1, sub * LANES + LANES - 1);
+            f2 = __shfl_sync(PODS_FULL_MASK, i2, sub * LANES + LANES - 1);
+            // Both ends are summed directly (lowest upward, highest downward): no split score is a
+            // difference of running totals, so equal splits score equal and nothing cancels.
+            double a1 = i1 - s1, a2 = i2 - s2;               // sum over positions below this lane's first
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int p = sl * E + e;
+                if (p <= m) { PL1[p] = a1; PL2[p] = a2; }
+                a1 += x[e];
+                a2 += x[e] * x[e];
+            }
+            if (sl == LANES - 1 && m == NPAD) { PL1[m] = a1; PL2[m] = a2; }   // position m does not exist: the total
+            double b1 = j1 - s1, b2 = j2 - s2;               // sum over positions above this lane's last
+            if (sl == LANES - 1 && n == NPAD) { SU1[m] = 0.0; SU2[m] = 0.0; }
+#pragma unroll
+            for (int e = E - 1; e >= 0; --e) {
+                const int p = sl * E + e;
+                b1 += x[e];
+                b2 += x[e] * x[e];
+                if (p >= n - m && p <= n) { SU1[p - (n - m)] = b1; SU2[p - (n - m)] = b2; }
+            }
+            __syncwarp();
+
+            // ---- 4. score the splits: m^2 Var = m * sum x^2 - (sum x)^2 ----------------------------
+            if (rule == PODS_RULE_MAXVAR && m < n) {
+                double best = -INFINITY;
+                int bestk = 0x7fffffff;
+                for (int k = sl; k <= m; k += LANES) {
+                    const double q1 = PL1[m - k] + SU1[m - k];
+                    const double q2 = PL2[m - k] + SU2[m - k];
+                    // separately rounded products (no fused multiply-add): equal sums give equal scores
+                    const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
+                    if (score > best || bestk == 0x7fffffff) { best = score; bestk = k; }
+                }
+#pragma unroll
+                for (int d = LANES >> 1; d > 0; d >>= 1) {
+                    const double ob = __shfl_xor_sync(PODS_FULL_MASK, best, d);
+                    const int ok = __shfl_xor_sync(PODS_FULL_MASK, bestk, d);
+                    if (ok != 0x7fffffff && (bestk == 0x7fffffff || ob > best || (ob == best && ok < bestk))) {
+                        best = ob;
+                        bestk = ok;
+                    }
+                }
+                kstar = __shfl_sync(PODS_FULL_MASK, bestk, sub * LANES);   // one verdict per group, even with NaN scores
+            }
+            k1 = PL1[m - kstar] + SU1[m - kstar];
+            k2 = PL2[m - kstar] + SU2[m - kstar];
+            __syncwarp();
+        }
+
+        // ---- 5. the two thresholds and how many of their ties are kept -------------------------------
+        const int nlo = m - kstar, nhi = kstar;
+        const uint32_t v_lo = key_at<LANES, E>(key, nlo > 0 ? nlo - 1 : 0, sub);
+        const uint32_t v_hi = key_at<LANES, E>(key, nhi > 0 ? n - nhi : 0, sub);
+        int c_less = 0, c_greater = 0, c_eq_hi = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const bool real = sl * E + e < n;
+            c_less += (real && key[e] < v_lo) ? 1 : 0;
+            c_greater += (real && key[e] > v_hi) ? 1 : 0;
+            c_eq_hi += (real && key[e] == v_hi) ? 1 : 0;
+        }
+        int packed = c_less | (c_greater << 10) | (c_eq_hi << 20);            // three counts <= 1023 in one word
+#pragma unroll
+        for (int d = LANES >> 1; d > 0; d >>= 1) packed += __shfl_xor_sync(PODS_FULL_MASK, packed, d);
+        const int need_lo = nlo - (packed & 1023);                           // rewards equal to v_lo to keep: the first by index
+        const int need_hi = nhi - ((packed >> 10) & 1023);                   // rewards equal to v_hi to keep: the last by index
+        const int first_hi = ((packed >> 20) & 1023) - need_hi;              // ... i.e. those from this rank on
+
+        // advantages: a = (x - S/c) / sigma with sigma^2 = (c Q - S^2) / (c d), d = c or c - 1
+        double s1 = k1, s2 = k2;
+        if (flags & PODS_FLAG_ADV_BEFORE) { s1 = f1; s2 = f2; }
+        const double cnt = (flags & PODS_FLAG_ADV_BEFORE) ? (double)n : (double)m;
+        const double den = (flags & PODS_FLAG_STD_SAMPLE) ? cnt - 1.0 : cnt;
+        const double J = __dsub_rn(__dmul_rn(cnt, s2), __dmul_rn(s1, s1));
+        const double inv_sigma_c = (J > 0.0 && den > 0.0) ? sqrt(den / (cnt * J)) : 0.0;   // 1 / (c sigma)
+
+        // ---- 6. emit in ascending original index ---------------------------------------------------
+        int written = 0, seen_lo = 0, seen_hi = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int i = e * LANES + sl;
+            const uint32_t ki = ordered_bits(orig[e]);
+            const bool in = i < n;
+            const bool eq_lo = in && nlo > 0 && ki == v_lo, eq_hi = in && nhi > 0 && ki == v_hi;
+            const uint32_t below = (1u << sl) - 1u;
+            const uint32_t b_lo = (__ballot_sync(PODS_FULL_MASK, eq_lo) >> (sub * LANES)) & GROUP_MASK;
+            const uint32_t b_hi = (__ballot_sync(PODS_FULL_MASK, eq_hi) >> (sub * LANES)) & GROUP_MASK;
+            const int rank_lo = seen_lo + __popc(b_lo & below), rank_hi = seen_hi + __popc(b_hi & below);
+            const bool take = in && ((nlo > 0 && ki < v_lo) || (eq_lo && rank_lo < need_lo) ||
+                                     (nhi > 0 && ki > v_hi) || (eq_hi && rank_hi >= first_hi));
+            const uint32_t b_take = (__ballot_sync(PODS_FULL_MASK, take) >> (sub * LANES)) & GROUP_MASK;
+            if (take && valid) {
+                const int off = written + __popc(b_take & below);
+                const double xi = (double)orig[e] - centre;
+                idx_out[g * (int64_t)m + off] = i;
+                adv_out[g * (int64_t)m + off] = (float)((xi * cnt - s1) * inv_sigma_c);
+            }
+            written += __popc(b_take);
+            seen_lo += __popc(b_lo);
+            seen_hi += __popc(b_hi);
+        }
+        if (valid && sl == 0 && k_out != nullptr) k_out[g] = kstar;
+        __syncwarp();
+    }
+}
+
+template <int LANES, int E>
+int launch_select_fast(const float* rewards, int64_t G, int n, int m, int rule, uint32_t flags, int32_t* idx,
+                       float* adv, int32_t* k_out, uint32_t* status, cudaStream_t stream) {
+    constexpr int GPW = 32 / LANES;
+    const size_t smem = (size_t)4 * (m + 1) * sizeof(double) * kSelectWarps * GPW;
+    auto kernel = pods_select_fast_kernel<LANES, E>;
+    if (smem > 48 * 1024)
+        PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t groups_per_cta = (int64_t)kSelectWarps * GPW;
+    const int64_t needed = (G + groups_per_cta - 1) / groups_per_cta;
+    const int64_t cap = (int64_t)pods_sm_count() * 16;
+    const int grid = (int)(needed < cap ? needed : cap);
+    kernel<<<grid, kSelectThreads, smem, stream>>>(rewards, G, n, m, rule, flags, idx, adv, k_out, status);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
 template <int LANES, int E>
 int launch_select(const float* rewards, int64_t G, int n, int m, int rule, uint64_t seed, uint32_t flags,
                   int32_t* idx, float* adv, int32_t* k_out, uint32_t* status, cudaStream_t stream) {
@@ -333,6 +590,19 @@ extern "C" int pods_select(const float* rewards, int64_t G, int32_t n, int32_t m
     if (rewards == nullptr || idx == nullptr || adv == nullptr) return PODS_ERR_INVALID_ARG;
     if (!pods_aligned(rewards, 4) || !pods_aligned(idx, 4) || !pods_aligned(adv, 4)) return PODS_ERR_INVALID_ARG;
     cudaStream_t s = pods_stream(stream);
+    if (rule == PODS_RULE_MAXVAR || rule == PODS_RULE_MAXREWARD) {
+#define PODS_SELECT_FAST(LANES, E) \
+    return launch_select_fast<LANES, E>(rewards, G, n, m, rule, flags, idx, adv, k_out, status, s)
+        if (n <= 8) PODS_SELECT_FAST(4, 2);
+        if (n <= 16) PODS_SELECT_FAST(4, 4);
+        if (n <= 32) PODS_SELECT_FAST(4, 8);
+        if (n <= 64) PODS_SELECT_FAST(8, 8);
+        if (n <= 128) PODS_SELECT_FAST(8, 16);
+        if (n <= 256) PODS_SELECT_FAST(16, 16);
+        if (n <= 512) PODS_SELECT_FAST(32, 16);
+        PODS_SELECT_FAST(32, 32);
+#undef PODS_SELECT_FAST
+    }
 #define PODS_SELECT_CASE(LANES, E) \
     return launch_select<LANES, E>(rewards, G, n, m, rule, seed, flags, idx, adv, k_out, status, s)
     if (n <= 8) PODS_SELECT_CASE(8, 1);
