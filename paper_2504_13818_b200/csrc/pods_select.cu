@@ -326,13 +326,12 @@ __device__ __forceinline__ uint32_t key_at(const uint32_t (&key)[E], int p, int 
 }
 
 template <int LANES, int E>
-__global__ void __launch_bounds__(kSelectThreads)
+__global__ void __launch_bounds__(kSelectThreads, E >= 32 ? 2 : 4)
 pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint32_t flags,
                         int32_t* __restrict__ idx_out, float* __restrict__ adv_out, int32_t* __restrict__ k_out,
                         uint32_t* status) {
     constexpr int NPAD = LANES * E;
     constexpr int GPW = 32 / LANES;                 // groups per warp
-    constexpr uint32_t GROUP_MASK = LANES == 32 ? 0xffffffffu : ((1u << LANES) - 1u);
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -341,6 +340,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
     double* PL2 = PL1 + (m + 1);
     double* SU1 = PL2 + (m + 1);                        // sum of the m-j highest, j = 0..m
     double* SU2 = SU1 + (m + 1);
+    const bool vec_rows = E % 4 == 0 && (n & 3) == 0 && (reinterpret_cast<uintptr_t>(rewards) & 15) == 0;
 
     const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
     for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
@@ -348,18 +348,35 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         const bool valid = g < G;
         const float* r_g = rewards + (valid ? g : 0) * (int64_t)n;
 
-        // ---- 1. load (coalesced: lane sl holds original indices e*LANES + sl) and key -----------
-        float orig[E];
-        uint32_t key[E];
+        // ---- 1. load and key: lane sl holds original indices sl*E .. sl*E+E-1 (okey keeps that order) ----
+        uint32_t okey[E];
         bool nonfinite = false;
+        if (vec_rows) {
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const int i = e * LANES + sl;
-            orig[e] = (i < n && valid) ? r_g[i] : 0.0f;
-            nonfinite |= !(fabsf(orig[e]) <= 3.402823466e38f);
-            key[e] = i < n ? ordered_bits(orig[e]) : 0xffffffffu;     // padding sorts last (with the NaNs, whose key it shares)
+            for (int e = 0; e < E; e += 4) {
+                const int i = sl * E + e;
+                float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (i < n && valid) v = *reinterpret_cast<const float4*>(r_g + i);
+                const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    nonfinite |= !(fabsf(f[c]) <= 3.402823466e38f);
+                    okey[e + c < E ? e + c : 0] = i < n ? ordered_bits(f[c]) : 0xffffffffu;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int i = sl * E + e;
+                const float r = (i < n && valid) ? r_g[i] : 0.0f;
+                nonfinite |= !(fabsf(r) <= 3.402823466e38f);
+                okey[e] = i < n ? ordered_bits(r) : 0xffffffffu;      // padding sorts last (with the NaNs, whose key it shares)
+            }
         }
         if (nonfinite && valid) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
+        uint32_t key[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) key[e] = okey[e];
 
         // ---- 2. bitonic sort of the keys over positions p = sl * E + e ------------------------------
 #pragma unroll
@@ -411,19 +428,18 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         // ---- 3. centred rewards and fp64 running sums over the sorted order ------------------------
         const uint32_t first = __shfl_sync(PODS_FULL_MASK, key[0], sub * LANES);
         const double centre = (double)from_ordered_bits(first);              // the group minimum
+        auto x_of = [&](uint32_t kk, int p) { return p < n ? (double)from_ordered_bits(kk) - centre : 0.0; };
         int kstar = rule == PODS_RULE_MAXREWARD ? m : 0;                      // m == n: every split is the whole group
         double k1 = 0.0, k2 = 0.0;                                            // sums of x and x^2 over the kept subset
         double f1 = 0.0, f2 = 0.0;                                            // ... and over the full group
         {
-            double x[E];
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const int p = sl * E + e;
-                x[e] = p < n ? (double)from_ordered_bits(key[e]) - centre : 0.0;
-            }
             double s1 = 0.0, s2 = 0.0;
 #pragma unroll
-            for (int e = 0; e < E; ++e) { s1 += x[e]; s2 += x[e] * x[e]; }
+            for (int e = 0; e < E; ++e) {
+                const double x = x_of(key[e], sl * E + e);
+                s1 += x;
+                s2 += x * x;
+            }
             double i1 = s1, i2 = s2;                         // inclusive scan over the lanes below
             double j1 = s1, j2 = s2;                         // inclusive scan over the lanes above
 #pragma unroll
@@ -435,27 +451,35 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
                 if (sl >= d) { i1 += t1; i2 += t2; }
                 if (sl + d < LANES) { j1 += u1; j2 += u2; }
             }
-            f1 = __shfl_sync(PODS_FULL_MASK, i1, sub * LANES + LANES - 1);
-            f2 = __shfl_sync(PODS_FULL_MASK, i2, sub * LANES + LANES - 1);
+            if (flags & PODS_FLAG_ADV_BEFORE) {
+                f1 = __shfl_sync(PODS_FULL_MASK, i1, sub * LANES + LANES - 1);
+                f2 = __shfl_sync(PODS_FULL_MASK, i2, sub * LANES + LANES - 1);
+            }
             // Both ends are summed directly (lowest upward, highest downward): no split score is a
             // difference of running totals, so equal splits score equal and nothing cancels.
             double a1 = i1 - s1, a2 = i2 - s2;               // sum over positions below this lane's first
+            if (sl * E <= m) {
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const int p = sl * E + e;
-                if (p <= m) { PL1[p] = a1; PL2[p] = a2; }
-                a1 += x[e];
-                a2 += x[e] * x[e];
+                for (int e = 0; e < E; ++e) {
+                    const int p = sl * E + e;
+                    if (p <= m) { PL1[p] = a1; PL2[p] = a2; }
+                    const double x = x_of(key[e], p);
+                    a1 += x;
+                    a2 += x * x;
+                }
+                if (sl == LANES - 1 && m == NPAD) { PL1[m] = a1; PL2[m] = a2; }   // position m does not exist: the total
             }
-            if (sl == LANES - 1 && m == NPAD) { PL1[m] = a1; PL2[m] = a2; }   // position m does not exist: the total
             double b1 = j1 - s1, b2 = j2 - s2;               // sum over positions above this lane's last
             if (sl == LANES - 1 && n == NPAD) { SU1[m] = 0.0; SU2[m] = 0.0; }
+            if (sl * E + E - 1 >= n - m) {
 #pragma unroll
-            for (int e = E - 1; e >= 0; --e) {
-                const int p = sl * E + e;
-                b1 += x[e];
-                b2 += x[e] * x[e];
-                if (p >= n - m && p <= n) { SU1[p - (n - m)] = b1; SU2[p - (n - m)] = b2; }
+                for (int e = E - 1; e >= 0; --e) {
+                    const int p = sl * E + e;
+                    const double x = x_of(key[e], p);
+                    b1 += x;
+                    b2 += x * x;
+                    if (p >= n - m && p <= n) { SU1[p - (n - m)] = b1; SU2[p - (n - m)] = b2; }
+                }
             }
             __syncwarp();
 
@@ -490,20 +514,32 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         const int nlo = m - kstar, nhi = kstar;
         const uint32_t v_lo = key_at<LANES, E>(key, nlo > 0 ? nlo - 1 : 0, sub);
         const uint32_t v_hi = key_at<LANES, E>(key, nhi > 0 ? n - nhi : 0, sub);
-        int c_less = 0, c_greater = 0, c_eq_hi = 0;
+        // counts over the ORIGINAL order (lane-major = index order), three 10-bit fields in one word:
+        // below v_lo | above v_hi | equal to v_lo | ... ; a group-wide inclusive scan gives totals and,
+        // per lane, how many ties precede it in index order
+        int c_less = 0, c_greater = 0, c_eqlo = 0, c_eqhi = 0;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             const bool real = sl * E + e < n;
-            c_less += (real && key[e] < v_lo) ? 1 : 0;
-            c_greater += (real && key[e] > v_hi) ? 1 : 0;
-            c_eq_hi += (real && key[e] == v_hi) ? 1 : 0;
+            c_less += (real && okey[e] < v_lo) ? 1 : 0;
+            c_greater += (real && okey[e] > v_hi) ? 1 : 0;
+            c_eqlo += (real && okey[e] == v_lo) ? 1 : 0;
+            c_eqhi += (real && okey[e] == v_hi) ? 1 : 0;
         }
-        int packed = c_less | (c_greater << 10) | (c_eq_hi << 20);            // three counts <= 1023 in one word
+        unsigned long long packed = (unsigned long long)c_less | ((unsigned long long)c_greater << 11) |
+                                    ((unsigned long long)c_eqlo << 22) | ((unsigned long long)c_eqhi << 33);
+        unsigned long long incl = packed;
 #pragma unroll
-        for (int d = LANES >> 1; d > 0; d >>= 1) packed += __shfl_xor_sync(PODS_FULL_MASK, packed, d);
-        const int need_lo = nlo - (packed & 1023);                           // rewards equal to v_lo to keep: the first by index
-        const int need_hi = nhi - ((packed >> 10) & 1023);                   // rewards equal to v_hi to keep: the last by index
-        const int first_hi = ((packed >> 20) & 1023) - need_hi;              // ... i.e. those from this rank on
+        for (int d = 1; d < LANES; d <<= 1) {
+            const unsigned long long t = __shfl_up_sync(PODS_FULL_MASK, incl, d, LANES);
+            if (sl >= d) incl += t;
+        }
+        const unsigned long long total = __shfl_sync(PODS_FULL_MASK, incl, sub * LANES + LANES - 1);
+        const unsigned long long before = incl - packed;
+        const int need_lo = nlo - (int)(total & 2047);                        // rewards equal to v_lo to keep: the first by index
+        const int need_hi = nhi - (int)((total >> 11) & 2047);                // rewards equal to v_hi to keep: the last by index
+        const int first_hi = (int)((total >> 33) & 2047) - need_hi;           // ... i.e. those from this rank on
+        int rank_lo = (int)((before >> 22) & 2047), rank_hi = (int)((before >> 33) & 2047);
 
         // advantages: a = (x - S/c) / sigma with sigma^2 = (c Q - S^2) / (c d), d = c or c - 1
         double s1 = k1, s2 = k2;
@@ -513,32 +549,40 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         const double J = __dsub_rn(__dmul_rn(cnt, s2), __dmul_rn(s1, s1));
         const double inv_sigma_c = (J > 0.0 && den > 0.0) ? sqrt(den / (cnt * J)) : 0.0;   // 1 / (c sigma)
 
-        // ---- 6. emit in ascending original index ---------------------------------------------------
-        int written = 0, seen_lo = 0, seen_hi = 0;
+        // ---- 6. which of my rewards are kept; their places in the output (ascending original index) ----
+        uint32_t take_bits = 0u;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            const int i = e * LANES + sl;
-            const uint32_t ki = ordered_bits(orig[e]);
-            const bool in = i < n;
+            const uint32_t ki = okey[e];
+            const bool in = sl * E + e < n;
             const bool eq_lo = in && nlo > 0 && ki == v_lo, eq_hi = in && nhi > 0 && ki == v_hi;
-            const uint32_t below = (1u << sl) - 1u;
-            const uint32_t b_lo = (__ballot_sync(PODS_FULL_MASK, eq_lo) >> (sub * LANES)) & GROUP_MASK;
-            const uint32_t b_hi = (__ballot_sync(PODS_FULL_MASK, eq_hi) >> (sub * LANES)) & GROUP_MASK;
-            const int rank_lo = seen_lo + __popc(b_lo & below), rank_hi = seen_hi + __popc(b_hi & below);
             const bool take = in && ((nlo > 0 && ki < v_lo) || (eq_lo && rank_lo < need_lo) ||
                                      (nhi > 0 && ki > v_hi) || (eq_hi && rank_hi >= first_hi));
-            const uint32_t b_take = (__ballot_sync(PODS_FULL_MASK, take) >> (sub * LANES)) & GROUP_MASK;
-            if (take && valid) {
-                const int off = written + __popc(b_take & below);
-                const double xi = (double)orig[e] - centre;
-                idx_out[g * (int64_t)m + off] = i;
-                adv_out[g * (int64_t)m + off] = (float)((xi * cnt - s1) * inv_sigma_c);
-            }
-            written += __popc(b_take);
-            seen_lo += __popc(b_lo);
-            seen_hi += __popc(b_hi);
+            take_bits |= take ? (1u << e) : 0u;
+            rank_lo += (in && ki == v_lo) ? 1 : 0;
+            rank_hi += (in && ki == v_hi) ? 1 : 0;
         }
-        if (valid && sl == 0 && k_out != nullptr) k_out[g] = kstar;
+        int my_takes = __popc(take_bits), off = my_takes;
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) {
+            const int t = __shfl_up_sync(PODS_FULL_MASK, off, d, LANES);
+            if (sl >= d) off += t;
+        }
+        off -= my_takes;
+        if (valid) {
+            int32_t* io = idx_out + g * (int64_t)m;
+            float* ao = adv_out + g * (int64_t)m;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                if ((take_bits >> e) & 1u) {
+                    const double xi = (double)from_ordered_bits(okey[e]) - centre;
+                    io[off] = sl * E + e;
+                    ao[off] = (float)((xi * cnt - s1) * inv_sigma_c);
+                    ++off;
+                }
+            }
+            if (sl == 0 && k_out != nullptr) k_out[g] = kstar;
+        }
         __syncwarp();
     }
 }
