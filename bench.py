@@ -110,6 +110,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(ms, device, world):
+    """The slowest rank's time: what a multi-process run reports (device-timed, MAX over ranks)."""
+    if world <= 1:
+        return float(ms)
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_per_step, steps, ms_total, world):
+    """Aggregate throughput of `world` independent replicas that each did the same work in ms_total."""
+    return world * units_per_rank_per_step * steps / (ms_total * 1e-3)
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -292,12 +307,7 @@ def run_ours(args):
     torch.cuda.cudart().cudaProfilerStop()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dev, world)
     status = binding.read_status(batch.status)
 
     # the dominant kernel: the fused loss rows kernel, timed per chunk launch on its own stream
@@ -316,7 +326,7 @@ def run_ours(args):
                 "rows_per_launch": batch.chunk}
 
     out = {
-        "metric": METRIC, "value": world * batch.T * args.steps / (ms_total * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": whole_job_value(batch.T, args.steps, ms_total, world), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 logits, f32 exp, f64 scalars",
         "data": "synthetic",
