@@ -637,10 +637,12 @@ extern "C" int pods_select(const float* rewards, int64_t G, int32_t n, int32_t m
     if (rule == PODS_RULE_MAXVAR || rule == PODS_RULE_MAXREWARD) {
 #define PODS_SELECT_FAST(LANES, E) \
     return launch_select_fast<LANES, E>(rewards, G, n, m, rule, flags, idx, adv, k_out, status, s)
-        if (n <= 8) PODS_SELECT_FAST(4, 2);
-        if (n <= 16) PODS_SELECT_FAST(4, 4);
-        if (n <= 32) PODS_SELECT_FAST(4, 8);
-        if (n <= 64) PODS_SELECT_FAST(8, 8);
+        // as many elements per lane as registers allow (16): compare-exchanges between registers cost one
+        // instruction per element, those between lanes a shuffle more, and the per-group scans get shorter
+        if (n <= 8) PODS_SELECT_FAST(2, 4);
+        if (n <= 16) PODS_SELECT_FAST(2, 8);
+        if (n <= 32) PODS_SELECT_FAST(2, 16);
+        if (n <= 64) PODS_SELECT_FAST(4, 16);
         if (n <= 128) PODS_SELECT_FAST(8, 16);
         if (n <= 256) PODS_SELECT_FAST(16, 16);
         if (n <= 512) PODS_SELECT_FAST(32, 16);
