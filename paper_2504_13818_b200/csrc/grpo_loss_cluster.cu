@@ -20,7 +20,7 @@
 //                        (m_w, sum_w) is handed to the exchange warp;
 //       back(i-1) grad   bf16(coef_w * e) by packed bf16 multiply-adds with coef_w split into two
 //                        bf16 terms (coef_w folds in 2^(ref_w - M log2e)), stored straight to global
-//                        memory with 128-bit streaming stores, the target entry then overwritten
+//                        memory with 128-bit stores, the target entry then overwritten
 //                        with g (1 - p) by the lane that stored its vector; the warp then arrives
 //                        on the stage's `done` barrier.
 //             front(i) runs before back(i-1), so the exchange of row i-1 has a whole sweep to finish.
@@ -445,7 +445,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 for (int k = 0; k < IT; ++k) {
                     const int j = lo + lane + 32 * k;
                     scale_vec(q[k], c_hi, c_lo);
-                    if (j < hi) __stcs(out + j, q[k]);
+                    if (j < hi) out[j] = q[k];
                 }
                 // the target entry, if it is in my slice: rewritten by the lane that stored its vector
                 if (tok_vec >= lo && tok_vec < hi && ((tok_vec - lo) & 31) == lane)

@@ -233,3 +233,20 @@ def test_cluster_path_token_in_every_segment_and_duplicate_maxima():
     b["logits"] = wl.f32_to_bf16_bits(x)
     b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
     _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+def test_cluster_path_without_reference_policy_and_single_rows():
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=16384, G=1, n=8, m=4, len_lo=3, len_hi=9, seed=41, beta=0.0)
+    b = build_batch(w)
+    want = oracle_loss(b)
+    _check(b, _gpu_loss(b, ref=False, mask=False), want)
+    _check(b, _gpu_loss(b, chunk_rows=1), want)            # one row per launch: a single cluster, one row each
+
+
+@pytest.mark.parametrize("V", [196608,      # twelve vectors per lane: the deepest register-held slice
+                               196616,      # one vector more: back to the general row kernel
+                               262144])
+def test_long_rows_on_both_sides_of_the_cluster_path_limit(V):
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=2, len_hi=5, seed=V % 97)
+    b = build_batch(w)
+    _check(b, _gpu_loss(b), oracle_loss(b))
