@@ -191,6 +191,15 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
                            double* loss_acc, float* logp, void* dlogits, int64_t ldd, uint32_t* status,
                            void* stream);
 
+/*
+ * pods_selftest_bounded_wait - diagnostic (the paper has no counterpart): one small kernel waits, with the
+ * same bounded poll loop the loss kernel uses for its barriers, on a barrier that nothing completes.
+ * After `polls` (1 .. 2^20) failed polls it must give up, OR PODS_STATUS_TIMEOUT into *status [dev]
+ * and return normally, leaving the context usable.  Shows that a lost signal ends in a status bit,
+ * not in a hang.
+ */
+int pods_selftest_bounded_wait(uint32_t polls, uint32_t* status, void* stream);
+
 /* Convert the fp64 accumulator of grpo_loss_chunk calls to the fp32 loss.  Both [dev]. */
 int grpo_loss_finalize(const double* loss_acc, float* loss, void* stream);
 

@@ -39,6 +39,7 @@ SIGNATURES = {
     "grpo_loss_fwd_bwd": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i32, _f32, _f32, _i64,
                                     _p, _p, _p, _i64, _p, _sz, _p, _p]),
     "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
+    "pods_selftest_bounded_wait": (C.c_int, [_u32, _p, _p]),
     "pods_host_step_create": (C.c_int, [_i64, _i32, _i32, _i64, _i64, _i32, _i64, _p]),
     "pods_host_step_run": (C.c_int, [_p, _p, _p, _p, _p, _p, _p, _i64, _f32, _f32, _i32, _u64, _u32,
                                      _p, _p, _p, _p, _p, _p]),
@@ -232,6 +233,12 @@ def grpo_loss_chunk_static(logits, tokens, old_logp, ref_logp, adv, seq_weight, 
                                        _dev(loss_acc, torch.float64, "loss_acc"), _dev(logp, torch.float32, "logp"),
                                        dp, ldd, _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_loss_chunk_static")
+
+
+def selftest_bounded_wait(polls, status):
+    """A wait on a barrier that nothing completes: must end by itself and set STATUS_TIMEOUT in ``status``."""
+    _check(load().pods_selftest_bounded_wait(polls, _dev(status, torch.int32, "status"), _stream()),
+           "pods_selftest_bounded_wait")
 
 
 def grpo_loss_finalize(loss_acc, loss):

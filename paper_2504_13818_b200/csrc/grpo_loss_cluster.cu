@@ -520,6 +520,15 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
     cluster_sync();                                    // no CTA leaves while a peer may still write its exchange slots
 }
 
+// One CTA, one mbarrier that nothing ever arrives on: the wait must give up after `polls` polls and
+// report it, and the kernel must end normally.
+__global__ void bounded_wait_selftest_kernel(uint32_t polls, uint32_t* status) {
+    __shared__ unsigned long long never;
+    if (threadIdx.x == 0) mbar_init(&never, 1);
+    __syncthreads();
+    if (!mbar_wait(&never, 0u, polls) && threadIdx.x == 0) pods_raise(status, PODS_STATUS_TIMEOUT);
+}
+
 struct ClusterPlan {
     int seg_vecs, n_stages;
     size_t smem;
@@ -588,6 +597,13 @@ int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
 }
 
 }  // namespace
+
+extern "C" int pods_selftest_bounded_wait(uint32_t polls, uint32_t* status, void* stream) {
+    if (status == nullptr || polls == 0 || polls > (1u << 20)) return PODS_ERR_INVALID_ARG;
+    bounded_wait_selftest_kernel<<<1, 64, 0, pods_stream(stream)>>>(polls, status);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
 
 namespace pods_loss {
 

@@ -250,3 +250,15 @@ def test_long_rows_on_both_sides_of_the_cluster_path_limit(V):
     w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=2, len_hi=5, seed=V % 97)
     b = build_batch(w)
     _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+def test_a_wait_that_nothing_ends_gives_up_with_a_status_bit_and_the_context_stays_usable():
+    """The loss kernel's barrier waits are bounded poll loops; the same loop on a barrier nobody completes
+    (no fault, no hang: the kernel just stops waiting) must raise STATUS_TIMEOUT, and the next call must work."""
+    status = binding.new_status()
+    binding.selftest_bounded_wait(1000, status)
+    torch.cuda.synchronize()
+    assert binding.read_status(status) == binding.STATUS_TIMEOUT
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=16384, G=1, n=8, m=4, len_lo=3, len_hi=6, seed=5)
+    b = build_batch(w)
+    _check(b, _gpu_loss(b), oracle_loss(b))
