@@ -262,3 +262,30 @@ def test_a_wait_that_nothing_ends_gives_up_with_a_status_bit_and_the_context_sta
     w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=16384, G=1, n=8, m=4, len_lo=3, len_hi=6, seed=5)
     b = build_batch(w)
     _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+def test_zero_length_rollouts_and_an_empty_batch():
+    """Rollouts with no tokens (cu_seqlens repeats a value) get weight 0 and own no row; T = 0 is a no-op with loss 0."""
+    for V in (520, 16384):
+        w = shrink(wl.WORKLOADS["c1_tiny"], G=2, n=8, m=4, V=V, len_lo=3, len_hi=7, seed=23)
+        b = build_batch(w)
+        # make kept rollouts 2 and 5 empty: drop their rows everywhere
+        cu = b["cu"].copy()
+        keep = np.ones(b["tokens"].shape[0], bool)
+        for i in (2, 5):
+            keep[cu[i]:cu[i + 1]] = False
+        lens = np.diff(cu)
+        lens[[2, 5]] = 0
+        b["cu"] = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        for key in ("tokens", "old", "ref", "mask", "logits"):
+            b[key] = np.ascontiguousarray(b[key][keep])
+        b["seq_of_row"] = oracle.seq_of_rows(b["cu"])
+        want = oracle_loss(b)
+        _check(b, _gpu_loss(b), want)
+    empty = torch.zeros((0, 16384), dtype=torch.bfloat16, device="cuda")
+    z32 = torch.zeros(0, dtype=torch.float32, device="cuda")
+    loss, logp, dl = binding.grpo_loss_fwd_bwd(empty, torch.zeros(0, dtype=torch.int32, device="cuda"), z32, z32,
+                                               torch.ones(2, device="cuda"), None, 0.2, 0.04,
+                                               torch.zeros(3, dtype=torch.int64, device="cuda"))
+    torch.cuda.synchronize()
+    assert float(loss.item()) == 0.0 and logp.numel() == 0 and dl.numel() == 0
