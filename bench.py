@@ -39,7 +39,7 @@ NCU_DRAM_BYTES_PER_ROW = 596500      # ncu capture of grpo_loss_cluster_kernel a
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_qwen_vocab")

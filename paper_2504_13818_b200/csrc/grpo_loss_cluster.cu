@@ -233,6 +233,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
     const int nvec = a.V / 8;
     const int seg0 = (int)rank * seg_vecs;                                   // first vector of my segment
     const int cnt = max(0, min(seg_vecs, nvec - seg0));                      // vectors in my segment
+    const int stage_vecs = (seg_vecs + 7) & ~7;                              // stages start on 128-byte lines
     const int64_t n_rows = cluster_id < a.T ? (a.T - cluster_id + n_clusters - 1) / n_clusters : 0;
     const bool has_ref = a.ref_logp != nullptr && a.beta != 0.0f;
 
@@ -262,7 +263,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 const uint4* src = reinterpret_cast<const uint4*>(a.logits + t * a.ldl) + seg0;
                 if (cnt > 0) {
                     mbar_expect_tx(&c.full[s], (uint32_t)cnt * 16u);
-                    uint4* dst = bufs + (size_t)s * seg_vecs;
+                    uint4* dst = bufs + (size_t)s * stage_vecs;
                     for (int v0 = 0; v0 < cnt; v0 += kPieceVecs)
                         bulk_load(dst + v0, src + v0, (uint32_t)min(kPieceVecs, cnt - v0) * 16u, &c.full[s]);
                 } else {
@@ -409,14 +410,14 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
         }
     } else {
         // =================================== consumer warps ===================================
-        const int per_warp = (cnt + kConsumerWarps - 1) / kConsumerWarps;
+        const int per_warp = ((cnt + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;     // slices start on 128-byte lines
         const int lo = min(cnt, warp * per_warp), hi = min(cnt, lo + per_warp);    // my slice of the segment
         const uint4 kNegInf4 = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
 
         // back(i): the gradient of row i over my slice, once the exchange warp has published its factors
         auto back = [&](int64_t i, int s) {
             const uint32_t xp = (uint32_t)(i & 1);
-            const uint4* const buf = bufs + (size_t)s * seg_vecs;
+            const uint4* const buf = bufs + (size_t)s * stage_vecs;
             const int64_t t = cluster_id + i * n_clusters;
             uint4* const out = reinterpret_cast<uint4*>(a.dlogits + t * a.ldd) + seg0;
             if (!mbar_wait(&c.ready[xp], (uint32_t)((i >> 1) & 1), timed_out ? 1u : kSpinLimit)) timed_out = true;
@@ -459,7 +460,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
         uint32_t parity = 0;
         for (int64_t i = 0; i < n_rows; ++i) {
             const uint32_t xp = (uint32_t)(i & 1);
-            uint4* const buf = bufs + (size_t)s * seg_vecs;
+            uint4* const buf = bufs + (size_t)s * stage_vecs;
 
             if (!mbar_wait(&c.full[s], parity, timed_out ? 1u : kSpinLimit)) timed_out = true;
 
@@ -539,8 +540,8 @@ struct ClusterPlan {
 // when three do not fit at all.
 bool plan_cluster(int nvec, int cl, ClusterPlan* p) {
     const size_t limit = 232448;
-    p->seg_vecs = (nvec + cl - 1) / cl;
-    const size_t seg_bytes = (size_t)p->seg_vecs * 16;
+    p->seg_vecs = ((nvec + cl - 1) / cl + 7) & ~7;                               // segments start on 128-byte lines of the row
+    const size_t seg_bytes = (size_t)((p->seg_vecs + 7) & ~7) * 16;               // a stage: the segment, padded to 128 bytes
     if (seg_bytes >= (1u << 20)) return false;
     for (int stages = kMaxStages; stages >= 2; --stages) {
         p->n_stages = stages;
@@ -585,7 +586,7 @@ int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
     ClusterPlan plan;
     if (!plan_cluster(a.V / 8, CL, &plan)) return PODS_OK;                 // does not fit: caller falls back
-    const int per_warp = (plan.seg_vecs + kConsumerWarps - 1) / kConsumerWarps;
+    const int per_warp = ((plan.seg_vecs + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;
     const int it = (per_warp + 31) / 32;
     if (it <= 2) return launch_cluster_it<CL, 2>(a, plan, stream, launched);
     if (it <= 4) return launch_cluster_it<CL, 4>(a, plan, stream, launched);
