@@ -329,7 +329,7 @@ def run_ours(args):
     out = {
         "metric": METRIC, "value": whole_job_value(batch.T, args.steps, ms_total, world), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 logits, f32 exp, f64 scalars",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "dtype_detail": "bf16 logits and gradients, f32 exponentials and sums, f64 per-row scalars",
         "data": "synthetic",
         "config": {"workload": w.name, "G": w.G, "n": w.n, "m": w.m, "V": w.V, "kept_tokens": batch.T,
                    "chunk_rows": batch.chunk, "l2": "inputs larger than L2 (logits %.1f GB per step)"
