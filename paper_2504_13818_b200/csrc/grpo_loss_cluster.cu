@@ -387,7 +387,8 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
             const double g = (in.w != 0.0) ? (double)a.grad_scale * in.w * dl : 0.0;
             if (lane < kConsumerWarps) {
                 // e^(x - M) = e_stored * 2^(ref_w - m_w log2e) * e^(m_w - M)
-                c.pub[xp].coef[lane] = (float)(-g * inv_z * ref_correction(my_m, my_m * kLog2e) * (double)my_scale);
+                c.pub[xp].coef[lane] = my_m == -INFINITY ? 0.0f     // a slice of -inf only: its e are all 0
+                                       : (float)(-g * inv_z * ref_correction(my_m, my_m * kLog2e) * (double)my_scale);
                 if (lane == 0) {
                     c.pub[xp].target = (float)(g * one_minus_p);
                     c.pub[xp].write_mode = (g != 0.0) ? 1 : 0;
@@ -479,7 +480,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
             const uint32_t key_w = __reduce_max_sync(PODS_FULL_MASK, (ordered16(m_t) << 16) | (uint32_t)(31 - lane));
             const float m_w = from_ordered16(key_w >> 16);
             const int owner = 31 - (int)(key_w & 0xffffu);               // lowest lane that holds an instance of m_w
-            const float ref_w = m_w * kLog2e;
+            const float ref_w = m_w == -INFINITY ? 0.0f : m_w * kLog2e;     // a slice of -inf only: every e is 0, not NaN
             // which of the owner's vectors holds it: the first k with that maximum (-1 on every other lane)
             int excl = -1;
             {

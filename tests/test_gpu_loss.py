@@ -289,3 +289,32 @@ def test_zero_length_rollouts_and_an_empty_batch():
                                                torch.zeros(3, dtype=torch.int64, device="cuda"))
     torch.cuda.synchronize()
     assert float(loss.item()) == 0.0 and logp.numel() == 0 and dl.numel() == 0
+
+
+@pytest.mark.parametrize("V", [4096, 32768])      # the general row kernel; the cluster path
+def test_masked_vocabulary_ranges_of_minus_infinity(V):
+    """Logits of -inf (ids a sampler has ruled out), scattered and as whole ranges longer than a warp's slice
+    and than a CTA's segment of the cluster path: probability and gradient exactly 0 there, nothing turns NaN."""
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=4, len_hi=8, seed=61)
+    b = build_batch(w)
+    x = wl.bf16_bits_to_f32(b["logits"])
+    rng = np.random.default_rng(7)
+    x[:, rng.uniform(size=V) < 0.1] = -np.inf            # scattered ids
+    lo, hi = (V * 5) // 8, (V * 13) // 16
+    x[:, lo:hi] = -np.inf                                # a range that covers whole warp slices and a whole segment
+    x[0, :] = -np.inf                                    # row 0: everything but one id
+    x[0, 77] = 1.5
+    rows = np.arange(x.shape[0])
+    tok = b["tokens"].copy()
+    tok[0] = 77
+    tok[1:] = np.where(np.isinf(x[rows[1:], tok[1:]]), 5, tok[1:])      # targets must be allowed ids
+    x[:, 5] = np.where(np.isinf(x[:, 5]), 0.25, x[:, 5])
+    b["tokens"] = tok.astype(np.int32)
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
+    want = oracle_loss(b)
+    assert np.isfinite(want["logp"]).all() and np.isfinite(want["dlogits"]).all()
+    got = _gpu_loss(b)
+    _check(b, got, want)
+    dl = wl.bf16_bits_to_f32(got[2])
+    assert np.isfinite(dl).all() and (dl[:, lo:hi] == 0).all()
