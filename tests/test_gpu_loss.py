@@ -318,3 +318,37 @@ def test_masked_vocabulary_ranges_of_minus_infinity(V):
     _check(b, got, want)
     dl = wl.bf16_bits_to_f32(got[2])
     assert np.isfinite(dl).all() and (dl[:, lo:hi] == 0).all()
+
+
+@pytest.mark.parametrize("V", [2048, 16384])
+def test_flat_rows_and_wide_logit_ranges(V):
+    """Rows whose logits are all equal (every element is the maximum; p = 1/V exactly) and rows whose range is
+    so wide that most probabilities underflow."""
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=5, len_hi=9, seed=67)
+    b = build_batch(w)
+    x = wl.bf16_bits_to_f32(b["logits"])
+    x[0, :] = 0.0
+    x[1, :] = -7.25
+    x[2, :] = 0.0
+    x[2, ::2] = -0.0                                      # the two zeros are one value
+    x[3:, :] *= 40.0                                      # spread of several hundred: e^(x - max) underflows
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
+    want = oracle_loss(b)
+    assert abs(want["logp"][0] + np.log(V)) < 1e-12 and abs(want["logp"][1] + np.log(V)) < 1e-12
+    got = _gpu_loss(b)
+    assert got[3] == 0
+    finite = np.isfinite(want["logp"]) & np.isfinite(want["g"])
+    assert finite[:3].all()
+    assert finite.all()
+    # log-probs of several hundred in magnitude: the fp32 output resolves them to ~3e-5, the bound stays 1e-3
+    assert np.abs(got[1] - want["logp"]).max() <= LOGP_ATOL
+    ulps = dlogits_ulp_error(got[2], want["dlogits"], gradient_slack(b, want))
+    # where the target holds all the mass but 1e-12, fp64 itself no longer resolves 1 - p (the oracle's plain
+    # log-sum-exp returns p = 1): the target's own entry is then left out, the rest of the row (zeros) is compared
+    unresolved = want["logp"] > -1e-12
+    assert 0 < unresolved.sum() < len(unresolved)
+    ulps[np.nonzero(unresolved)[0], b["tokens"][unresolved]] = 0.0
+    assert ulps.max() <= DLOGITS_ULPS
+    got_target = wl.bf16_bits_to_f32(got[2])[np.nonzero(unresolved)[0], b["tokens"][unresolved]]
+    assert (np.abs(got_target) < 1e-15).all()
