@@ -7,8 +7,9 @@
  * Conventions for every call
  *   - Pointers marked [dev] are device pointers on the current CUDA device, [host] are host
  *     pointers.  The caller owns every buffer; the library allocates no device memory and
- *     keeps no state between calls (except pods_host_step_*, which says what it allocates, and
- *     grpo_loss_chunk_static, which says what it holds).
+ *     keeps no state between calls (except pods_host_step_*, which says what it allocates,
+ *     grpo_loss_chunk_static, which says what it holds, and one tuning value, see
+ *     pods_set_loss_cluster_min_vocab).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
  *     enqueue work and return; outputs are valid once the stream has reached that point.
  *   - The return value is a pods_status.  Errors that the host can see (sizes, null or
@@ -190,6 +191,14 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
                            int64_t T_chunk, int32_t V, float eps, float beta, float grad_scale,
                            double* loss_acc, float* logp, void* dlogits, int64_t ldd, uint32_t* status,
                            void* stream);
+
+/*
+ * pods_set_loss_cluster_min_vocab - tuning knob (the paper has no counterpart): grpo_loss_chunk runs rows of
+ * V >= min_vocab (V % 8 == 0, 16-byte aligned rows) on the cluster-resident kernel and shorter rows on the
+ * general row kernel.  The default, 57344, is the measured cross-over on B200; values below 2048 are raised to
+ * 2048.  Process-wide; returns the previous value.  Results of either kernel meet the same tolerances.
+ */
+int32_t pods_set_loss_cluster_min_vocab(int32_t min_vocab);
 
 /*
  * pods_selftest_bounded_wait - diagnostic (the paper has no counterpart): one small kernel waits, with the

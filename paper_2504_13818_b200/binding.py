@@ -40,6 +40,7 @@ SIGNATURES = {
                                     _p, _p, _p, _i64, _p, _sz, _p, _p]),
     "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
     "pods_selftest_bounded_wait": (C.c_int, [_u32, _p, _p]),
+    "pods_set_loss_cluster_min_vocab": (_i32, [_i32]),
     "pods_host_step_create": (C.c_int, [_i64, _i32, _i32, _i64, _i64, _i32, _i64, _p]),
     "pods_host_step_run": (C.c_int, [_p, _p, _p, _p, _p, _p, _p, _i64, _f32, _f32, _i32, _u64, _u32,
                                      _p, _p, _p, _p, _p, _p]),
@@ -233,6 +234,11 @@ def grpo_loss_chunk_static(logits, tokens, old_logp, ref_logp, adv, seq_weight, 
                                        _dev(loss_acc, torch.float64, "loss_acc"), _dev(logp, torch.float32, "logp"),
                                        dp, ldd, _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_loss_chunk_static")
+
+
+def set_loss_cluster_min_vocab(min_vocab) -> int:
+    """Rows of V >= min_vocab take the cluster-resident loss kernel; returns the previous setting."""
+    return int(load().pods_set_loss_cluster_min_vocab(int(min_vocab)))
 
 
 def selftest_bounded_wait(polls, status):

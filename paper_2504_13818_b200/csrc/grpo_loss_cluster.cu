@@ -607,13 +607,23 @@ extern "C" int pods_selftest_bounded_wait(uint32_t polls, uint32_t* status, void
     return PODS_OK;
 }
 
+// Rows shorter than this go to the general row kernel: per row the cluster path pays a fixed price (the
+// exchange across the cluster, a pipeline stage per row), which only long rows repay.  Measured cross-over on
+// B200: the row kernel wins up to V = 49152 (3.9 against 3.4 TB/s), the cluster path from 65536 on (4.4 against 4.1).
+static int32_t g_cluster_min_vocab = 57344;
+
+extern "C" int32_t pods_set_loss_cluster_min_vocab(int32_t min_vocab) {
+    const int32_t v = min_vocab < 2048 ? 2048 : min_vocab;
+    return __atomic_exchange_n(&g_cluster_min_vocab, v, __ATOMIC_RELAXED);
+}
+
 namespace pods_loss {
 
 // Runs the chunk on the cluster path if the row shape allows it (16-byte aligned rows, V a multiple
 // of 8 and large enough to be worth a cluster, segments that fit in shared memory).
 int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
-    if (!a.vec_ok || a.V % 8 != 0 || a.V < 16384) return PODS_OK;
+    if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
     return launch_cluster<8>(a, stream, launched);
 }
 

@@ -16,6 +16,16 @@ from parity import (CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, assert_loss_close, bui
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["default", "cluster path from V = 2048"])
+def _both_loss_kernels(request):
+    """Every test runs twice: with the library's own choice between its two loss kernels, and with the
+    cluster-resident kernel forced on every vocabulary it can take (V >= 2048, V % 8 == 0, aligned rows)."""
+    previous = binding.set_loss_cluster_min_vocab(2048) if request.param != "default" else None
+    yield
+    if previous is not None:
+        binding.set_loss_cluster_min_vocab(previous)
+
+
 def _t(a, dtype=None):
     t = torch.from_numpy(np.ascontiguousarray(a))
     return (t if dtype is None else t.view(dtype)).cuda()
