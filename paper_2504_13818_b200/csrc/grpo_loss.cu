@@ -279,6 +279,151 @@ __global__ void loss_zero_kernel(double* loss_acc) { *loss_acc = 0.0; }
 
 __global__ void loss_finalize_kernel(const double* loss_acc, float* loss) { *loss = (float)*loss_acc; }
 
+
+// ---------------------------------------------------------------------------------------------
+// Row-tile kernel for short rows (V <= 4096, V % 8 == 0, 16-byte aligned rows).
+// ---------------------------------------------------------------------------------------------
+// A row of a small vocabulary is only a few KB: one CTA per row leaves most of its threads idle and
+// pays the fp64 scalar terms once per row on a single thread.  Here a CTA of eight warps takes a tile
+// of R rows (R * V * 2 bytes <= 64 KB of shared memory); one WARP owns a whole row:
+//   A  row -> registers with 128-bit loads, packed maxima, warp arg-max, e = 2^(x log2e - ref) summed
+//      with one instance of the maximum left out, bf16(e) parked in the tile;
+//   B  the first R threads of the CTA evaluate the fp64 scalar terms of one row each, side by side;
+//   C  each warp turns its rows' e into bf16(coef e) and stores them, then fixes the target entry.
+// HBM sees one read and one write per element; the exponential is taken once.
+constexpr int kTileWarps = 8;
+constexpr int kTileMaxRows = 64;
+constexpr int kTileBytes = 64 * 1024;
+
+template <int IT>
+__global__ void __launch_bounds__(kTileWarps * 32)
+grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
+    extern __shared__ __align__(16) uint4 tile[];
+    __shared__ float s_mx[kTileMaxRows], s_sum[kTileMaxRows], s_coef[kTileMaxRows], s_target[kTileMaxRows];
+    __shared__ int s_mode[kTileMaxRows], s_tok[kTileMaxRows];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = a.V / 8;
+    const uint4 neg_inf4 = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+
+    for (int64_t tile0 = (int64_t)blockIdx.x * rows_per_tile; tile0 < a.T; tile0 += (int64_t)gridDim.x * rows_per_tile) {
+        const int n_rows = (int)(a.T - tile0 < rows_per_tile ? a.T - tile0 : rows_per_tile);
+
+        // ---- A: statistics of my rows; e parked in the tile --------------------------------------------
+        for (int r = warp; r < n_rows; r += kTileWarps) {
+            const uint4* row4 = reinterpret_cast<const uint4*>(a.logits + (tile0 + r) * a.ldl);
+            uint4 q[IT];
+#pragma unroll
+            for (int k = 0; k < IT; ++k) {
+                const int j = lane + 32 * k;
+                q[k] = j < nvec ? row4[j] : neg_inf4;
+            }
+            uint32_t pm[4] = {kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair};
+#pragma unroll
+            for (int k = 0; k < IT; ++k) max_vec(pm, q[k]);
+            const uint32_t pmax = max_bf16x2(max_bf16x2(pm[0], pm[1]), max_bf16x2(pm[2], pm[3]));
+            const float m_t = fmaxf(bf16_lo(pmax), bf16_hi(pmax)) + 0.0f;             // -0 -> +0
+            const uint32_t key_w = __reduce_max_sync(PODS_FULL_MASK, (ordered16(m_t) << 16) | (uint32_t)(31 - lane));
+            const float mx = from_ordered16(key_w >> 16);
+            const int owner = 31 - (int)(key_w & 0xffffu);               // lowest lane that holds an instance of the maximum
+            const float ref = mx == -INFINITY ? 0.0f : mx * kLog2e;
+            int excl = -1;                                               // the owner's first vector that holds it
+            if (lane == owner) {
+#pragma unroll
+                for (int k = IT - 1; k >= 0; --k)
+                    if (vec_max(q[k]) == mx) excl = k;
+            }
+            float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < IT; ++k) {
+                const int j = lane + 32 * k;
+                const float part = (k == excl) ? exp_sum_excluding(q[k], ref, mx) : 0.0f;
+                const float sum = exp_vec_inplace(q[k], ref);
+                if (k & 1) s1 += (k == excl) ? part : sum; else s0 += (k == excl) ? part : sum;
+                if (j < nvec) tile[(size_t)r * nvec + j] = q[k];
+            }
+            float sw = s0 + s1;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) sw += __shfl_xor_sync(PODS_FULL_MASK, sw, d);
+            if (lane == 0) { s_mx[r] = mx; s_sum[r] = sw; }
+        }
+        __syncthreads();
+
+        // ---- B: the scalar terms, one row per thread ---------------------------------------------------------
+        if (tid < n_rows) {
+            const int64_t t = tile0 + tid;
+            int tok = a.tokens[t];
+            if (tok < 0 || tok >= a.V) { tok = 0; pods_raise(a.status, PODS_STATUS_TOKEN_RANGE); }
+            const float x_tok = __uint_as_float((uint32_t)a.logits[t * a.ldl + tok] << 16);   // before phase C stores this row in place
+            const float mx = s_mx[tid];
+            const double corr = ref_correction(mx, mx * kLog2e);
+            const RowInputs in = load_row_inputs(a, t);
+            const RowScalars r = row_scalars(a, in, x_tok, mx, (double)s_sum[tid] * corr);
+            a.logp[t] = (float)r.logp;
+            a.row_loss[t] = r.weighted_loss;
+            s_coef[tid] = (float)(-r.g / r.Z * corr);
+            s_target[tid] = (float)(r.g * r.one_minus_p);
+            s_mode[tid] = (r.g != 0.0) ? 1 : 0;
+            s_tok[tid] = tok;
+        }
+        __syncthreads();
+
+        // ---- C: the gradient rows ---------------------------------------------------------------------------
+        for (int r = warp; r < n_rows; r += kTileWarps) {
+            uint4* out = reinterpret_cast<uint4*>(a.dlogits + (tile0 + r) * a.ldd);
+            if (s_mode[r] == 0) {
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                for (int j = lane; j < nvec; j += 32) out[j] = z;
+                continue;
+            }
+            const float coef = s_coef[r];
+            const uint16_t hi16 = to_bf16_bits(coef);
+            const uint16_t lo16 = to_bf16_bits(coef - __uint_as_float((uint32_t)hi16 << 16));
+            const uint32_t c_hi = (uint32_t)hi16 * 0x10001u, c_lo = (uint32_t)lo16 * 0x10001u;
+#pragma unroll
+            for (int k = 0; k < IT; ++k) {
+                const int j = lane + 32 * k;
+                if (j < nvec) {
+                    uint4 e = tile[(size_t)r * nvec + j];
+                    scale_vec(e, c_hi, c_lo);
+                    out[j] = e;
+                }
+            }
+            const int tok = s_tok[r];
+            if (((tok >> 3) & 31) == lane)                               // rewritten by the lane that stored its vector
+                reinterpret_cast<uint16_t*>(out)[tok] = to_bf16_bits(s_target[r]);
+        }
+        __syncthreads();                                                 // the tile and the row slots are reused
+    }
+}
+
+template <int IT>
+int launch_tile(const RowArgs& a, cudaStream_t s) {
+    const int nvec = a.V / 8;
+    int rows = kTileBytes / (nvec * 16);
+    rows = rows > kTileMaxRows ? kTileMaxRows : rows & ~(kTileWarps - 1);
+    const size_t smem = (size_t)rows * nvec * 16;
+    auto kernel = grpo_loss_tile_kernel<IT>;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t tiles = (a.T + rows - 1) / rows;
+    const int64_t cap = (int64_t)pods_sm_count() * 3;
+    kernel<<<(unsigned)(tiles < cap ? tiles : cap), kTileWarps * 32, smem, s>>>(a, rows);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
+// Short rows on the row-tile kernel; *launched says whether the shape was taken.
+int launch_grpo_loss_tile(const RowArgs& a, cudaStream_t s, bool* launched) {
+    *launched = false;
+    if (!a.vec_ok || a.V % 8 != 0 || a.V > 4096) return PODS_OK;
+    *launched = true;
+    const int it = (a.V / 8 + 31) / 32;
+    if (it <= 1) return launch_tile<1>(a, s);
+    if (it <= 2) return launch_tile<2>(a, s);
+    if (it <= 4) return launch_tile<4>(a, s);
+    if (it <= 8) return launch_tile<8>(a, s);
+    return launch_tile<16>(a, s);
+}
+
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
@@ -337,6 +482,14 @@ extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* t
     const int rc_cluster = launch_grpo_loss_cluster(a, s, &on_cluster_path);
     if (rc_cluster != PODS_OK) return rc_cluster;
     if (on_cluster_path) {
+        loss_reduce_kernel<<<1, 1024, 0, s>>>(a.row_loss, T_chunk, loss_acc);
+        PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+        return PODS_OK;
+    }
+    bool on_tile_path = false;
+    const int rc_tile = launch_grpo_loss_tile(a, s, &on_tile_path);
+    if (rc_tile != PODS_OK) return rc_tile;
+    if (on_tile_path) {
         loss_reduce_kernel<<<1, 1024, 0, s>>>(a.row_loss, T_chunk, loss_acc);
         PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
         return PODS_OK;

@@ -72,6 +72,67 @@ __device__ __forceinline__ int argmax_key_pos(unsigned long long k) {
     return 0x7fffffff - (int)(uint32_t)(k & 0xffffffffu);
 }
 
+// ---- pieces of the register-held sweeps shared by the cluster-resident and the row-tile kernels ----
+
+// bf16 value (as fp32, -0 already folded into +0) -> 16-bit key whose unsigned order is the order of the values.
+__device__ __forceinline__ uint32_t ordered16(float v) {
+    const uint32_t u = __float_as_uint(v) >> 16;
+    return (u & 0x8000u) ? (~u & 0xffffu) : (u | 0x8000u);
+}
+__device__ __forceinline__ float from_ordered16(uint32_t o) {
+    const uint32_t u = (o & 0x8000u) ? (o & 0x7fffu) : (~o & 0xffffu);
+    return __uint_as_float(u << 16);
+}
+
+// e = 2^(x log2e - ref) for the eight values of a vector: returns their sum, leaves bf16(e) in q.
+__device__ __forceinline__ float exp_vec_inplace(uint4& q, float ref) {
+    const float e0 = ex2_approx(fmaf(bf16_lo(q.x), kLog2e, -ref)), e1 = ex2_approx(fmaf(bf16_hi(q.x), kLog2e, -ref));
+    const float e2 = ex2_approx(fmaf(bf16_lo(q.y), kLog2e, -ref)), e3 = ex2_approx(fmaf(bf16_hi(q.y), kLog2e, -ref));
+    const float e4 = ex2_approx(fmaf(bf16_lo(q.z), kLog2e, -ref)), e5 = ex2_approx(fmaf(bf16_hi(q.z), kLog2e, -ref));
+    const float e6 = ex2_approx(fmaf(bf16_lo(q.w), kLog2e, -ref)), e7 = ex2_approx(fmaf(bf16_hi(q.w), kLog2e, -ref));
+    q.x = pack_bf16x2(e0, e1);
+    q.y = pack_bf16x2(e2, e3);
+    q.z = pack_bf16x2(e4, e5);
+    q.w = pack_bf16x2(e6, e7);
+    return ((e0 + e1) + (e2 + e3)) + ((e4 + e5) + (e6 + e7));
+}
+
+// Sum over the vector's values of 2^(x log2e - ref), the first one equal to mx left out.
+static __device__ __noinline__ float exp_sum_excluding(uint4 q, float ref, float mx) {
+    const float v[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                        bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+    float s = 0.0f;
+    bool skipped = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const bool skip = !skipped && v[i] == mx;
+        skipped |= skip;
+        s += skip ? 0.0f : ex2_approx(fmaf(v[i], kLog2e, -ref));
+    }
+    return s;
+}
+
+// bf16(e * (c_hi + c_lo)) for two packed bf16 e: the small term first, then one fused rounding.
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t e, uint32_t c_hi, uint32_t c_lo) {
+    uint32_t t, o;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(t) : "r"(e), "r"(c_lo));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o) : "r"(e), "r"(c_hi), "r"(t));
+    return o;
+}
+__device__ __forceinline__ void scale_vec(uint4& q, uint32_t c_hi, uint32_t c_lo) {
+    q.x = scale_bf16x2(q.x, c_hi, c_lo);
+    q.y = scale_bf16x2(q.y, c_hi, c_lo);
+    q.z = scale_bf16x2(q.z, c_hi, c_lo);
+    q.w = scale_bf16x2(q.w, c_hi, c_lo);
+}
+
+__device__ __forceinline__ void max_vec(uint32_t (&pm)[4], const uint4& q) {
+    pm[0] = max_bf16x2(pm[0], q.x);
+    pm[1] = max_bf16x2(pm[1], q.y);
+    pm[2] = max_bf16x2(pm[2], q.z);
+    pm[3] = max_bf16x2(pm[3], q.w);
+}
+
 // Everything the objective needs for one row besides the logits, gathered by the cluster path's
 // preparation kernel: 32 bytes, read as two 16-byte vectors.
 struct __align__(16) RowPrep {
