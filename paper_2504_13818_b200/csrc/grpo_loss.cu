@@ -2,6 +2,10 @@
 // respect to the bf16 logits, fused: per row the softmax statistics and the target log-prob, the
 // scalar loss terms, then the gradient row.
 //
+// grpo_loss_chunk picks one of three kernels by the row shape: the cluster-resident pipeline
+// (grpo_loss_cluster.cu) for long aligned rows, the row-tile kernel below for short aligned rows, and
+// the general row kernel for everything else (any V, any pitch or alignment).
+//
 // Row kernel (one CTA per row at a time, persistent over rows), three uniform sweeps of the row:
 //   max   128-bit loads from HBM, packed bf16x2 maxima; each thread remembers where its maximum
 //         was; a block arg-max gives the row maximum M and the position of its first instance;
