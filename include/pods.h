@@ -195,8 +195,8 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
 /*
  * pods_set_loss_cluster_min_vocab - tuning knob (the paper has no counterpart): grpo_loss_chunk runs rows of
  * V >= min_vocab (V % 8 == 0, 16-byte aligned rows) on the cluster-resident kernel and shorter rows on the
- * general row kernel.  The default, 57344, is the measured cross-over on B200; values below 2048 are raised to
- * 2048.  Process-wide; returns the previous value.  Results of either kernel meet the same tolerances.
+ * row-tile (V <= 4096) or the general row kernel.  The default, 8192, is the measured cross-over on B200; values
+ * below 2048 are raised to 2048.  Process-wide; returns the previous value.  Results of either kernel meet the same tolerances.
  */
 int32_t pods_set_loss_cluster_min_vocab(int32_t min_vocab);
 

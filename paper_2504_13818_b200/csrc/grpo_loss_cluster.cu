@@ -548,10 +548,11 @@ extern "C" int pods_selftest_bounded_wait(uint32_t polls, uint32_t* status, void
     return PODS_OK;
 }
 
-// Rows shorter than this go to the general row kernel: per row the cluster path pays a fixed price (the
-// exchange across the cluster, a pipeline stage per row), which only long rows repay.  Measured cross-over on
-// B200: the row kernel wins up to V = 49152 (3.9 against 3.4 TB/s), the cluster path from 65536 on (4.4 against 4.1).
-static int32_t g_cluster_min_vocab = 57344;
+// Rows shorter than this go to the row-tile or the general row kernel: per row the cluster path pays a
+// fixed price (a pipeline stage and an exchange per row), which very short rows do not repay.  Measured on
+// B200 with the cluster size chosen below: 4.4 TB/s at V = 8192 (the row kernel: 3.8), 5.7-6.0 from 12288 on;
+// 2.8 at V = 4096, where the row-tile kernel does 3.6.
+static int32_t g_cluster_min_vocab = 8192;
 
 extern "C" int32_t pods_set_loss_cluster_min_vocab(int32_t min_vocab) {
     const int32_t v = min_vocab < 2048 ? 2048 : min_vocab;
@@ -565,6 +566,13 @@ namespace pods_loss {
 int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
     if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
+    // as few CTAs per row as leave room for the full ring with two CTAs per SM: fewer partners to exchange
+    // with, longer slices per warp, and small clusters fill the GPU better than clusters of eight
+    ClusterPlan p;
+    const size_t half_sm = 233472 / 2 - 1024;
+    if (plan_cluster(a.V / 8, 1, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<1>(a, stream, launched);
+    if (plan_cluster(a.V / 8, 2, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<2>(a, stream, launched);
+    if (plan_cluster(a.V / 8, 4, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<4>(a, stream, launched);
     return launch_cluster<8>(a, stream, launched);
 }
 
