@@ -566,13 +566,20 @@ namespace pods_loss {
 int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
     if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
-    // as few CTAs per row as leave room for the full ring with two CTAs per SM: fewer partners to exchange
-    // with, longer slices per warp, and small clusters fill the GPU better than clusters of eight
+    // as few CTAs per row (1 .. 8, any number) as leave room for the full ring with two CTAs per SM: fewer
+    // partners to exchange with, longer slices per warp, and small clusters fill the GPU better than large ones
     ClusterPlan p;
     const size_t half_sm = 233472 / 2 - 1024;
-    if (plan_cluster(a.V / 8, 1, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<1>(a, stream, launched);
-    if (plan_cluster(a.V / 8, 2, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<2>(a, stream, launched);
-    if (plan_cluster(a.V / 8, 4, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<4>(a, stream, launched);
+#define PODS_TRY_CLUSTER(CL) \
+    if (plan_cluster(a.V / 8, CL, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<CL>(a, stream, launched)
+    PODS_TRY_CLUSTER(1);
+    PODS_TRY_CLUSTER(2);
+    PODS_TRY_CLUSTER(3);
+    PODS_TRY_CLUSTER(4);
+    PODS_TRY_CLUSTER(5);
+    PODS_TRY_CLUSTER(6);
+    PODS_TRY_CLUSTER(7);
+#undef PODS_TRY_CLUSTER
     return launch_cluster<8>(a, stream, launched);
 }
 
