@@ -53,3 +53,12 @@ def test_binding_refuses_host_tensors():
     import torch
     with pytest.raises(binding.PodsError):
         binding.pods_select(torch.zeros(2, 4), 2)
+
+
+def test_cluster_vocabulary_limit_is_a_process_wide_setting_with_a_floor():
+    lib = binding.load()
+    default = lib.pods_set_loss_cluster_min_vocab(100000)
+    assert default == 8192
+    assert lib.pods_set_loss_cluster_min_vocab(5) == 100000       # values below 2048 are raised to 2048
+    assert lib.pods_set_loss_cluster_min_vocab(default) == 2048
+    assert lib.pods_set_loss_cluster_min_vocab(default) == default
