@@ -362,3 +362,36 @@ def test_flat_rows_and_wide_logit_ranges(V):
     assert ulps.max() <= DLOGITS_ULPS
     got_target = wl.bf16_bits_to_f32(got[2])[np.nonzero(unresolved)[0], b["tokens"][unresolved]]
     assert (np.abs(got_target) < 1e-15).all()
+
+
+def test_repeated_launches_are_bit_identical_on_every_kernel_in_and_out_of_place():
+    """A few hundred launches per shape (row-tile kernel, row kernel, clusters of 1, 3 and 8 CTAs): any race in
+    the pipelines or the exchange would show as a differing bit or a status bit sooner or later."""
+    dev = torch.device("cuda")
+    g = torch.Generator(device=dev)
+    g.manual_seed(11)
+    for V, T in [(1024, 700), (6000, 300), (12288, 900), (40960, 500), (151936, 150)]:
+        logits = (torch.randn((T, V), generator=g, device=dev) * 3).to(torch.bfloat16)
+        tokens = torch.randint(0, V, (T,), generator=g, device=dev, dtype=torch.int32)
+        cu = torch.linspace(0, T, 9, device=dev).long()
+        lt = wl.library_logp(logits, tokens)
+        old = lt + 0.05 * torch.randn(T, generator=g, device=dev)
+        ref = lt + 0.05 * torch.randn(T, generator=g, device=dev)
+        adv = torch.randn(8, generator=g, device=dev)
+        sw = binding.grpo_seq_weights(None, cu)
+        ws = torch.empty(binding.grpo_loss_chunk_workspace_bytes(T), dtype=torch.uint8, device=dev)
+
+        def run(in_place):
+            src = logits.clone() if in_place else logits
+            dl = src if in_place else torch.empty_like(logits)
+            acc = torch.zeros(1, dtype=torch.float64, device=dev)
+            logp = torch.empty(T, device=dev)
+            status = binding.new_status(dev)
+            binding.grpo_loss_chunk(src, tokens, old, ref, adv, sw, cu, 0, None, 0.2, 0.04, acc, logp, dl, ws, status=status)
+            return dl, logp, acc, status
+
+        dl0, logp0, acc0, _ = run(False)
+        for i in range(120):
+            dl, logp, acc, status = run(bool(i & 1))
+            assert torch.equal(dl.view(torch.int16), dl0.view(torch.int16)) and torch.equal(logp, logp0)
+            assert float(acc.item()) == float(acc0.item()) and binding.read_status(status) == 0
