@@ -6,6 +6,9 @@
 // so HBM sees exactly one read and one write per element and every other access is to shared
 // memory.  A CTA is eight consumer warps, one producer warp and one exchange warp that meet only
 // through mbarriers, over a ring of NS segment buffers; no warp ever waits at a CTA-wide barrier.
+// CL is chosen per launch: the smallest of 1 .. 8 whose segment leaves room for the ring with two
+// CTAs per SM (8 for a 152 K vocabulary, 1 for 16 K): small clusters have fewer partners to wait for
+// and leave fewer CTA slots of the GPU empty.
 //
 //   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
 //             pieces counted on the stage's `full` barrier, never multicast); as soon as the
