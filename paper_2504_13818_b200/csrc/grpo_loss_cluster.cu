@@ -6,9 +6,11 @@
 // so HBM sees exactly one read and one write per element and every other access is to shared
 // memory.  A CTA is eight consumer warps, one producer warp and one exchange warp that meet only
 // through mbarriers, over a ring of NS segment buffers; no warp ever waits at a CTA-wide barrier.
-// CL is chosen per launch: the smallest of 1 .. 8 whose segment leaves room for the ring with two
-// CTAs per SM (8 for a 152 K vocabulary, 1 for 16 K): small clusters have fewer partners to wait for
-// and leave fewer CTA slots of the GPU empty.
+// CL is chosen per launch: the smallest of 1 .. 10, 12, 16 whose segment leaves room for the
+// ring with two CTAs per SM (8 for a 152 K vocabulary, 1 for 16 K, 16 for 256 K): small clusters have
+// fewer partners to wait for and leave fewer CTA slots of the GPU empty (cluster placement fills 296
+// slots with clusters of 1 or 2, 264 with 8, 224 with 16).  Sizes above 8 are non-portable cluster
+// sizes, which the launch asks for explicitly.
 //
 //   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
 //             pieces counted on the stage's `full` barrier, never multicast); as soon as the
@@ -57,10 +59,12 @@ constexpr int kProducerWarp = kConsumerWarps;       // warp 8
 constexpr int kExchangeWarp = kConsumerWarps + 1;   // warp 9
 constexpr int kThreads = kConsumers + 64;
 constexpr int kMaxStages = 3;
-constexpr int kMaxCluster = 8;
-constexpr int kMaxSlots = kMaxCluster * kConsumerWarps;   // (m_w, sum_w) pairs per row
 constexpr int kPieceVecs = 512;               // 16-byte vectors per bulk load (8 KB)
-constexpr int kCtrlBytes = 1408;              // barriers, exchange slots and row scalars ahead of the buffers
+// (m_w, sum_w) slots per row parity: 64 serve clusters of up to 8 CTAs, 128 the larger ones (up to 16, which
+// the launch has to ask for as a non-portable cluster size)
+__host__ __device__ constexpr int slot_count(int cl) { return cl <= 8 ? 64 : 128; }
+// barriers, row scalars and exchange slots ahead of the buffers
+__host__ __device__ constexpr int ctrl_bytes(int cl) { return cl <= 8 ? 1408 : 2432; }
 constexpr uint32_t kSpinLimit = 1u << 24;     // polls of one barrier or slot before giving up (a fraction of a second)
 constexpr uint32_t kSuspendNs = 1000;         // upper bound on the time one poll may suspend the thread
 
@@ -77,17 +81,19 @@ struct RowPublish {                           // what back(i) needs, per row par
     int pad;
 };
 
+template <int SLOTS>
 struct Ctrl {
     unsigned long long full[kMaxStages];      // producer -> consumers: the stage's segment has landed
     unsigned long long done[kMaxStages];      // consumers -> producer: the stage has been read for the last time
     unsigned long long sumdone[2];            // consumers -> exchange: the CTA's pairs of the row are in `part`
     unsigned long long ready[2];              // exchange -> consumers: `pub` of the row is valid
     Pair part[2][kConsumerWarps];
-    unsigned long long xslot[2][kMaxSlots];   // slot [parity][8 rank + warp] is written by CTA `rank` of the cluster:
-                                              // (sum_w bits) << 32 | (ordered bf16 m_w) << 16 | tag of the row
     RowPublish pub[2];
+    unsigned long long xslot[2][SLOTS];       // slot [parity][8 rank + warp] is written by CTA `rank` of the cluster:
+                                              // (sum_w bits) << 32 | (ordered bf16 m_w) << 16 | tag of the row
 };
-static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+static_assert(sizeof(Ctrl<slot_count(8)>) <= ctrl_bytes(8) && sizeof(Ctrl<slot_count(16)>) <= ctrl_bytes(16),
+              "control block too large");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -168,8 +174,9 @@ template <int CL, int IT>
 __global__ void __launch_bounds__(kThreads, 2)
 grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages) {
     extern __shared__ __align__(128) unsigned char smem[];
-    Ctrl& c = *reinterpret_cast<Ctrl*>(smem);
-    uint4* const bufs = reinterpret_cast<uint4*>(smem + kCtrlBytes);
+    constexpr int kSlots = slot_count(CL);
+    Ctrl<kSlots>& c = *reinterpret_cast<Ctrl<kSlots>*>(smem);
+    uint4* const bufs = reinterpret_cast<uint4*>(smem + ctrl_bytes(CL));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_rank();
@@ -181,7 +188,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
     const int64_t n_rows = cluster_id < a.T ? (a.T - cluster_id + n_clusters - 1) / n_clusters : 0;
     const bool has_ref = a.ref_logp != nullptr && a.beta != 0.0f;
 
-    if (tid < 2 * kMaxSlots) (&c.xslot[0][0])[tid] = 0ull;         // tag 0 is no row's tag
+    if (tid < 2 * kSlots) (&c.xslot[0][0])[tid] = 0ull;            // tag 0 is no row's tag
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&c.full[s], 1);                  // the copy issuer, with the byte count
@@ -260,29 +267,31 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 for (uint32_t peer = (uint32_t)lane >> 3; peer < (uint32_t)CL; peer += 4)
                     push_word(peer_address(&c.xslot[xp][rank * kConsumerWarps + w], peer), word);
             }
-            // lane l collects slots l and l + 32: polls until both carry the row's tag
-            unsigned long long w0 = tag, w1 = tag;
+            // lane l collects slots l, l + 32, ...: polls until all carry the row's tag
+            constexpr int NW = (CL * kConsumerWarps + 31) / 32;
+            unsigned long long word[NW];
             {
                 const uint32_t limit = timed_out ? 1u : kSpinLimit;
                 uint32_t it = 0;
                 for (;;) {
-                    if (lane < n_slots) w0 = poll_word(&c.xslot[xp][lane]);
-                    if (lane + 32 < n_slots) w1 = poll_word(&c.xslot[xp][lane + 32]);
-                    const bool ok = (w0 & 0xffffull) == tag && (w1 & 0xffffull) == tag;
+                    bool ok = true;
+#pragma unroll
+                    for (int q = 0; q < NW; ++q) {
+                        word[q] = tag;
+                        if (lane + 32 * q < n_slots) word[q] = poll_word(&c.xslot[xp][lane + 32 * q]);
+                        ok = ok && (word[q] & 0xffffull) == tag;
+                    }
                     if (__all_sync(PODS_FULL_MASK, ok)) break;
                     if (++it >= limit) { timed_out = true; break; }
                 }
             }
-            // lane l holds slots l and l + 32
-            Pair p0, p1;
-            p0.key = (uint32_t)w0 & 0xffff0000u;
-            p0.sum = __uint_as_float((uint32_t)(w0 >> 32));
-            p1.key = (uint32_t)w1 & 0xffff0000u;
-            p1.sum = __uint_as_float((uint32_t)(w1 >> 32));
             // the row maximum; among equal maxima the lowest slot's instance is the one left out of the sums
-            const uint32_t cand0 = lane < n_slots ? ((p0.key & 0xffff0000u) | (uint32_t)(0xffff - lane)) : 0u;
-            const uint32_t cand1 = lane + 32 < n_slots ? ((p1.key & 0xffff0000u) | (uint32_t)(0xffff - lane - 32)) : 0u;
-            const uint32_t best = __reduce_max_sync(PODS_FULL_MASK, max(cand0, cand1));
+            uint32_t cand = 0u;
+#pragma unroll
+            for (int q = 0; q < NW; ++q)
+                if (lane + 32 * q < n_slots)
+                    cand = max(cand, ((uint32_t)word[q] & 0xffff0000u) | (uint32_t)(0xffff - lane - 32 * q));
+            const uint32_t best = __reduce_max_sync(PODS_FULL_MASK, cand);
             const float mx = from_ordered16(best >> 16);
             const int owner_slot = 0xffff - (int)(best & 0xffffu);
             // the exponentials of the scalar terms need only the maximum: three lanes, three calls at once
@@ -291,32 +300,32 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
             const double part = exp(lane == 0 ? xr - (double)in.old_logp : (lane == 1 ? (double)in.ref_logp - xr : xr));
             // sum_w is relative to ref_w: bring it to the row maximum; every slice but the owner's gets back
             // the instance of its own maximum that it left out
-            const float m0 = from_ordered16(p0.key >> 16), m1 = from_ordered16(p1.key >> 16);
-            float scale0 = 0.0f, scale1 = 0.0f;
+            float m_q[NW], scale_q[NW];
             double contrib = 0.0;
-            if (lane < n_slots && m0 != -INFINITY) {
-                scale0 = ex2_approx((m0 - mx) * kLog2e);
-                const double tr = (double)p0.sum * ref_correction(m0, m0 * kLog2e);
-                contrib += (lane == owner_slot) ? tr : (tr + 1.0) * (double)scale0;
-            }
-            if (lane + 32 < n_slots && m1 != -INFINITY) {
-                scale1 = ex2_approx((m1 - mx) * kLog2e);
-                const double tr = (double)p1.sum * ref_correction(m1, m1 * kLog2e);
-                contrib += (lane + 32 == owner_slot) ? tr : (tr + 1.0) * (double)scale1;
+#pragma unroll
+            for (int q = 0; q < NW; ++q) {
+                m_q[q] = from_ordered16((uint32_t)word[q] >> 16);
+                scale_q[q] = 0.0f;
+                if (lane + 32 * q < n_slots && m_q[q] != -INFINITY) {
+                    scale_q[q] = ex2_approx((m_q[q] - mx) * kLog2e);
+                    const double tr = (double)__uint_as_float((uint32_t)(word[q] >> 32)) * ref_correction(m_q[q], m_q[q] * kLog2e);
+                    contrib += (lane + 32 * q == owner_slot) ? tr : (tr + 1.0) * (double)scale_q[q];
+                }
             }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) contrib += __shfl_xor_sync(PODS_FULL_MASK, contrib, d);
             const double zp = contrib;                                         // Z - 1
             const double Z = 1.0 + zp;
             const double inv_z = 1.0 / Z;
-            // the factors of this CTA's own slices: slot rank * 8 + w sits in lane (rank * 8 + w) % 32
+            // the factors of this CTA's own slices: slot rank * 8 + w sits in word (slot / 32) of lane (slot % 32)
             const int my_slot = (int)rank * kConsumerWarps + (lane & 7);
-            const float sc_lo = __shfl_sync(PODS_FULL_MASK, scale0, my_slot & 31);
-            const float sc_hi = __shfl_sync(PODS_FULL_MASK, scale1, my_slot & 31);
-            const float mw_lo = __shfl_sync(PODS_FULL_MASK, m0, my_slot & 31);
-            const float mw_hi = __shfl_sync(PODS_FULL_MASK, m1, my_slot & 31);
-            const float my_scale = my_slot < 32 ? sc_lo : sc_hi;
-            const float my_m = my_slot < 32 ? mw_lo : mw_hi;
+            float my_scale = 0.0f, my_m = 0.0f;
+#pragma unroll
+            for (int q = 0; q < NW; ++q) {
+                const float sc = __shfl_sync(PODS_FULL_MASK, scale_q[q], my_slot & 31);
+                const float mm = __shfl_sync(PODS_FULL_MASK, m_q[q], my_slot & 31);
+                if ((my_slot >> 5) == q) { my_scale = sc; my_m = mm; }
+            }
             const double adv = (double)in.adv;
             const double rho = __shfl_sync(PODS_FULL_MASK, part, 0) * inv_z;
             const double ed = has_ref ? __shfl_sync(PODS_FULL_MASK, part, 1) * Z : 1.0;
@@ -475,6 +484,8 @@ __global__ void bounded_wait_selftest_kernel(uint32_t polls, uint32_t* status) {
     if (!mbar_wait(&never, 0u, polls) && threadIdx.x == 0) pods_raise(status, PODS_STATUS_TIMEOUT);
 }
 
+constexpr size_t kHalfSmBytes = 233472 / 2 - 1024;      // what a CTA may hold for two of them to share an SM
+
 struct ClusterPlan {
     int seg_vecs, n_stages;
     size_t smem;
@@ -490,7 +501,7 @@ bool plan_cluster(int nvec, int cl, ClusterPlan* p) {
     if (seg_bytes >= (1u << 20)) return false;
     for (int stages = kMaxStages; stages >= 2; --stages) {
         p->n_stages = stages;
-        p->smem = kCtrlBytes + (size_t)stages * seg_bytes;
+        p->smem = (size_t)ctrl_bytes(cl) + (size_t)stages * seg_bytes;
         if (p->smem <= limit) return true;
     }
     return false;
@@ -501,6 +512,7 @@ int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t
     ClusterPlan plan = plan_in;
     auto kernel = grpo_loss_cluster_kernel<CL, IT>;
     PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
+    if (CL > 8) PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -525,21 +537,36 @@ int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t
     return PODS_OK;
 }
 
-// IT = vectors per lane of a consumer warp's slice, rounded up to the next instantiated depth.
+// IT = vectors per lane of a consumer warp's slice.  Every depth a cluster size can be chosen with is
+// instantiated (unused lanes of the last vector cost as much as used ones, so rounding IT up to an even
+// number cost up to 15 % where it applied).  A size CL > 1 is only chosen when CL - 1 CTAs do not fit,
+// so its segments are at least (CL-1)/CL of the largest one that fits and its depths start at kMinIt;
+// all sizes but the largest are bounded by the two-CTAs-per-SM segment (depth 10), the largest by the
+// register file (depth 12, with a ring of two stages, or one CTA per SM, for its longest segments).
+template <int CL> constexpr int kMinIt = CL == 1 ? 1 : CL == 2 ? 5 : CL == 3 ? 7 : 8;
+template <int CL> constexpr int kMaxIt = CL == 16 ? 12 : 10;
+
+template <int CL, int IT>
+int launch_cluster_from(int it, const RowArgs& a, const ClusterPlan& plan, cudaStream_t stream, bool* launched) {
+    if (it <= IT) return launch_cluster_it<CL, IT>(a, plan, stream, launched);
+    if constexpr (IT < kMaxIt<CL>) return launch_cluster_from<CL, IT + 1>(it, a, plan, stream, launched);
+    return PODS_OK;                                                        // rows too long for the register-held slices
+}
+
 template <int CL>
 int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
     ClusterPlan plan;
     if (!plan_cluster(a.V / 8, CL, &plan)) return PODS_OK;                 // does not fit: caller falls back
+    // segments too long for two CTAs per SM with the full ring: two CTAs with a ring of two beat one CTA
+    // with a ring of three (measured, V = 155648 .. 196608: +3 %)
+    const size_t seg_bytes = (size_t)((plan.seg_vecs + 7) & ~7) * 16;
+    if (plan.smem > kHalfSmBytes && ctrl_bytes(CL) + 2 * seg_bytes <= kHalfSmBytes) {
+        plan.n_stages = 2;
+        plan.smem = ctrl_bytes(CL) + 2 * seg_bytes;
+    }
     const int per_warp = ((plan.seg_vecs + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;
-    const int it = (per_warp + 31) / 32;
-    if (it <= 2) return launch_cluster_it<CL, 2>(a, plan, stream, launched);
-    if (it <= 4) return launch_cluster_it<CL, 4>(a, plan, stream, launched);
-    if (it <= 6) return launch_cluster_it<CL, 6>(a, plan, stream, launched);
-    if (it <= 8) return launch_cluster_it<CL, 8>(a, plan, stream, launched);
-    if (it <= 10) return launch_cluster_it<CL, 10>(a, plan, stream, launched);
-    if (it <= 12) return launch_cluster_it<CL, 12>(a, plan, stream, launched);
-    return PODS_OK;                                                        // rows too long for the register-held slices
+    return launch_cluster_from<CL, kMinIt<CL>>((per_warp + 31) / 32, a, plan, stream, launched);
 }
 
 }  // namespace
@@ -569,12 +596,11 @@ namespace pods_loss {
 int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
     *launched = false;
     if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
-    // as few CTAs per row (1 .. 8, any number) as leave room for the full ring with two CTAs per SM: fewer
-    // partners to exchange with, longer slices per warp, and small clusters fill the GPU better than large ones
+    // as few CTAs per row as leave room for the full ring with two CTAs per SM: fewer partners to exchange
+    // with, longer slices per warp, and small clusters fill the GPU better than large ones
     ClusterPlan p;
-    const size_t half_sm = 233472 / 2 - 1024;
 #define PODS_TRY_CLUSTER(CL) \
-    if (plan_cluster(a.V / 8, CL, &p) && p.n_stages == kMaxStages && p.smem <= half_sm) return launch_cluster<CL>(a, stream, launched)
+    if (plan_cluster(a.V / 8, CL, &p) && p.n_stages == kMaxStages && p.smem <= kHalfSmBytes) return launch_cluster<CL>(a, stream, launched)
     PODS_TRY_CLUSTER(1);
     PODS_TRY_CLUSTER(2);
     PODS_TRY_CLUSTER(3);
@@ -582,8 +608,12 @@ int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launch
     PODS_TRY_CLUSTER(5);
     PODS_TRY_CLUSTER(6);
     PODS_TRY_CLUSTER(7);
+    PODS_TRY_CLUSTER(8);
+    PODS_TRY_CLUSTER(9);
+    PODS_TRY_CLUSTER(10);
+    PODS_TRY_CLUSTER(12);             // 11 and 13 to 15 place badly (231 and at most 221 of the 296 CTA slots)
 #undef PODS_TRY_CLUSTER
-    return launch_cluster<8>(a, stream, launched);
+    return launch_cluster<16>(a, stream, launched);
 }
 
 }  // namespace pods_loss

@@ -253,13 +253,46 @@ def test_cluster_path_without_reference_policy_and_single_rows():
     _check(b, _gpu_loss(b, chunk_rows=1), want)            # one row per launch: a single cluster, one row each
 
 
-@pytest.mark.parametrize("V", [196608,      # twelve vectors per lane: the deepest register-held slice
-                               196616,      # one vector more: back to the general row kernel
-                               262144])
-def test_long_rows_on_both_sides_of_the_cluster_path_limit(V):
+@pytest.mark.parametrize("V", [163840,      # nine CTAs per row: the first non-portable cluster size
+                               180224,      # ten
+                               196608,      # twelve
+                               262144,      # sixteen
+                               301056,      # sixteen, the longest segment with three stages and two CTAs per SM
+                               393216,      # sixteen, twelve vectors per lane: the deepest register-held slice
+                               393224])     # one vector more: back to the general row kernel
+def test_long_rows_up_to_and_beyond_the_cluster_path_limit(V):
     w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=2, len_hi=5, seed=V % 97)
     b = build_batch(w)
     _check(b, _gpu_loss(b), oracle_loss(b))
+
+
+def test_long_rows_on_the_two_stage_ring_with_several_rows_per_cluster():
+    """V = 327680 over 16 CTAs: segments of 40 KB, too long for three stages with two CTAs per SM, so the ring
+    has two stages; 14 such clusters are resident at most, so with > 80 rows every stage is reused several times."""
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=327680, G=2, n=8, m=4, len_lo=10, len_hi=18, seed=163)
+    b = build_batch(w)
+    assert b["tokens"].shape[0] > 80
+    got = _gpu_loss(b)
+    _check(b, got, oracle_loss(b))
+    assert _gpu_loss(b, in_place=True)[2].tobytes() == got[2].tobytes()
+
+
+def test_large_clusters_with_many_rows_masks_and_duplicate_maxima():
+    """V = 176128 over ten CTAs (34.4 KB segments), several rows per cluster, some rows masked, maxima repeated across segments."""
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=176128, G=2, n=8, m=4, len_lo=10, len_hi=18, seed=176)
+    b = build_batch(w)
+    T = b["tokens"].shape[0]
+    assert T > 80
+    rng = np.random.default_rng(11)
+    b["mask"] = (rng.uniform(size=T) < 0.8).astype(np.uint8)
+    x = wl.bf16_bits_to_f32(b["logits"])
+    x[0, [3, 60000, 120000, 176127]] = 15.0                # the maximum in four different CTAs' segments
+    x[1, b["tokens"][1]] += 18.0                           # nearly certain of its token
+    b["logits"] = wl.f32_to_bf16_bits(x)
+    b["old"], b["ref"] = wl.make_old_ref(w, wl.host_logp_tilde(b["logits"], b["tokens"]))
+    got = _gpu_loss(b)
+    _check(b, got, oracle_loss(b))
+    assert (got[2][b["mask"] == 0] == 0).all()
 
 
 def test_a_wait_that_nothing_ends_gives_up_with_a_status_bit_and_the_context_stays_usable():
