@@ -7,10 +7,11 @@
 // memory.  A CTA is eight consumer warps, one producer warp and one exchange warp that meet only
 // through mbarriers, over a ring of NS segment buffers; no warp ever waits at a CTA-wide barrier.
 // CL is chosen per launch: the smallest of 1 .. 10, 12, 16 whose segment leaves room for the
-// ring with two CTAs per SM (8 for a 152 K vocabulary, 1 for 16 K, 16 for 256 K): small clusters have
+// ring with two CTAs per SM (8 for a 128 K vocabulary, 1 for 16 K, 16 for 256 K): small clusters have
 // fewer partners to wait for and leave fewer CTA slots of the GPU empty (cluster placement fills 296
 // slots with clusters of 1 or 2, 264 with 8, 224 with 16).  Sizes above 8 are non-portable cluster
-// sizes, which the launch asks for explicitly.
+// sizes, which the launch asks for explicitly.  Where the smallest size needs the deepest register slices,
+// the next size is taken instead if it keeps more slice registers busy across the GPU (9 for 152 K).
 //
 //   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
 //             pieces counted on the stage's `full` barrier, never multicast); as soon as the
@@ -543,8 +544,17 @@ int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t
 // so its segments are at least (CL-1)/CL of the largest one that fits and its depths start at kMinIt;
 // all sizes but the largest are bounded by the two-CTAs-per-SM segment (depth 10), the largest by the
 // register file (depth 12, with a ring of two stages, or one CTA per SM, for its longest segments).
-template <int CL> constexpr int kMinIt = CL == 1 ? 1 : CL == 2 ? 5 : CL == 3 ? 7 : 8;
+// A size may also be chosen in place of the previous one at depth 10 (see pick_cluster), which lowers
+// the first depth of sizes 3, 4 and 16 by one.
+template <int CL> constexpr int kMinIt = CL == 1 ? 1 : CL == 2 ? 5 : CL == 3 ? 6 : (CL == 4 || CL == 16) ? 7 : 8;
 template <int CL> constexpr int kMaxIt = CL == 16 ? 12 : 10;
+constexpr int kDeepestPairedIt = 10;          // the deepest slices whose segment still fits twice per SM
+
+// vectors per lane of a consumer warp's slice of a segment: slices start on 128-byte lines
+int slice_depth(int seg_vecs) {
+    const int per_warp = ((seg_vecs + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;
+    return (per_warp + 31) / 32;
+}
 
 template <int CL, int IT>
 int launch_cluster_from(int it, const RowArgs& a, const ClusterPlan& plan, cudaStream_t stream, bool* launched) {
@@ -565,8 +575,69 @@ int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
         plan.n_stages = 2;
         plan.smem = ctrl_bytes(CL) + 2 * seg_bytes;
     }
-    const int per_warp = ((plan.seg_vecs + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;
-    return launch_cluster_from<CL, kMinIt<CL>>((per_warp + 31) / 32, a, plan, stream, launched);
+    return launch_cluster_from<CL, kMinIt<CL>>(slice_depth(plan.seg_vecs), a, plan, stream, launched);
+}
+
+// CTAs of this kernel that are resident at once when launched as clusters of CL with two CTAs per SM
+// (cluster placement leaves some of the 2 x SMs slots empty, how many depends on CL); -1 if the query fails.
+// Asked once per device.
+template <int CL>
+int resident_ctas() {
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    int v = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED);
+    if (v != 0) return v;
+    auto kernel = grpo_loss_cluster_kernel<CL, kDeepestPairedIt>;
+    v = -1;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(CL, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kHalfSmBytes;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHalfSmBytes) == cudaSuccess &&
+        (CL <= 8 || cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) &&
+        cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0)
+        v = n * CL;
+    else
+        (void)cudaGetLastError();
+    __atomic_store_n(&cached[dev], v, __ATOMIC_RELAXED);
+    return v;
+}
+
+// Launches on clusters of CL if the row's segments fit the full ring twice per SM; false if they do not.
+// At the deepest slices (depth 10) the next size NEXT takes over when it promises more: resident CTAs
+// x the share of the slice registers that hold data.  Measured, 2 GiB of logits: V = 129280 and 131072
+// 8 CTAs per row instead of 7 +3 %, 151936 and 152064 9 instead of 8 +2 %; at lower depths the same
+// product picked the slower size more often than not (40960, 49152, 86016, 100352), so there the smaller
+// size stays.
+template <int CL, int NEXT>
+bool pick_cluster(const RowArgs& a, cudaStream_t stream, bool* launched, int* rc) {
+    const int nvec = a.V / 8;
+    ClusterPlan p;
+    if (!(plan_cluster(nvec, CL, &p) && p.n_stages == kMaxStages && p.smem <= kHalfSmBytes)) return false;
+    if constexpr (NEXT != 0) {
+        ClusterPlan q;
+        if (slice_depth(p.seg_vecs) == kDeepestPairedIt && plan_cluster(nvec, NEXT, &q) && q.n_stages == kMaxStages &&
+            q.smem <= kHalfSmBytes) {
+            const int dq = slice_depth(q.seg_vecs) < kMinIt<NEXT> ? kMinIt<NEXT> : slice_depth(q.seg_vecs);
+            const double here = (double)resident_ctas<CL>() * nvec / ((double)CL * kDeepestPairedIt);
+            const double next = (double)resident_ctas<NEXT>() * nvec / ((double)NEXT * dq);
+            if (here > 0.0 && next > here) {
+                *rc = launch_cluster<NEXT>(a, stream, launched);
+                return true;
+            }
+        }
+    }
+    *rc = launch_cluster<CL>(a, stream, launched);
+    return true;
 }
 
 }  // namespace
@@ -597,22 +668,16 @@ int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launch
     *launched = false;
     if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
     // as few CTAs per row as leave room for the full ring with two CTAs per SM: fewer partners to exchange
-    // with, longer slices per warp, and small clusters fill the GPU better than large ones
-    ClusterPlan p;
-#define PODS_TRY_CLUSTER(CL) \
-    if (plan_cluster(a.V / 8, CL, &p) && p.n_stages == kMaxStages && p.smem <= kHalfSmBytes) return launch_cluster<CL>(a, stream, launched)
-    PODS_TRY_CLUSTER(1);
-    PODS_TRY_CLUSTER(2);
-    PODS_TRY_CLUSTER(3);
-    PODS_TRY_CLUSTER(4);
-    PODS_TRY_CLUSTER(5);
-    PODS_TRY_CLUSTER(6);
-    PODS_TRY_CLUSTER(7);
-    PODS_TRY_CLUSTER(8);
-    PODS_TRY_CLUSTER(9);
-    PODS_TRY_CLUSTER(10);
-    PODS_TRY_CLUSTER(12);             // 11 and 13 to 15 place badly (231 and at most 221 of the 296 CTA slots)
-#undef PODS_TRY_CLUSTER
+    // with, longer slices per warp, and small clusters fill the GPU better than large ones; 11 and 13 to 15
+    // place badly (231 and at most 221 of the 296 CTA slots of a B200)
+    int rc = PODS_OK;
+    if (pick_cluster<1, 2>(a, stream, launched, &rc) || pick_cluster<2, 3>(a, stream, launched, &rc) ||
+        pick_cluster<3, 4>(a, stream, launched, &rc) || pick_cluster<4, 5>(a, stream, launched, &rc) ||
+        pick_cluster<5, 6>(a, stream, launched, &rc) || pick_cluster<6, 7>(a, stream, launched, &rc) ||
+        pick_cluster<7, 8>(a, stream, launched, &rc) || pick_cluster<8, 9>(a, stream, launched, &rc) ||
+        pick_cluster<9, 10>(a, stream, launched, &rc) || pick_cluster<10, 12>(a, stream, launched, &rc) ||
+        pick_cluster<12, 16>(a, stream, launched, &rc))
+        return rc;
     return launch_cluster<16>(a, stream, launched);
 }
 
