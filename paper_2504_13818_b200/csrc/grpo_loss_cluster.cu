@@ -632,7 +632,7 @@ bool pick_cluster(const RowArgs& a, cudaStream_t stream, bool* launched, int* rc
             const double next = (double)resident_ctas<NEXT>() * nvec / ((double)NEXT * dq);
             if (here > 0.0 && next > here) {
                 *rc = launch_cluster<NEXT>(a, stream, launched);
-                return true;
+                if (*rc != PODS_OK || *launched) return true;
             }
         }
     }
