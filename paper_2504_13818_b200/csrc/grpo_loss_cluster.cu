@@ -258,7 +258,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
             in.token = (int)nx1.z;
             if (i + 1 < n_rows) { nx0 = prep4[2 * (t + n_clusters)]; nx1 = prep4[2 * (t + n_clusters) + 1]; }
             if (!mbar_wait(&c.sumdone[xp], xparity, timed_out ? 1u : kSpinLimit)) timed_out = true;
-            // lane l pushes pair (l % 8) of this CTA to peers l / 8 and l / 8 + 4
+            // lane l pushes pair (l % 8) of this CTA to peers l / 8, l / 8 + 4, l / 8 + 8, ...
             const unsigned long long tag = (unsigned long long)((i + 1) & 0xffff);
             {
                 const int w = lane & 7;
@@ -540,8 +540,8 @@ int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t
 
 // IT = vectors per lane of a consumer warp's slice.  Every depth a cluster size can be chosen with is
 // instantiated (unused lanes of the last vector cost as much as used ones, so rounding IT up to an even
-// number cost up to 15 % where it applied).  A size CL > 1 is only chosen when CL - 1 CTAs do not fit,
-// so its segments are at least (CL-1)/CL of the largest one that fits and its depths start at kMinIt;
+// number cost up to 15 % where it applied).  A size is only chosen when the size before it does not fit,
+// so its segments are at least that share of the largest one that fits and its depths start at kMinIt;
 // all sizes but the largest are bounded by the two-CTAs-per-SM segment (depth 10), the largest by the
 // register file (depth 12, with a ring of two stages, or one CTA per SM, for its longest segments).
 // A size may also be chosen in place of the previous one at depth 10 (see pick_cluster), which lowers
