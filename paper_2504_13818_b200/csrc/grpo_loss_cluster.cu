@@ -14,7 +14,7 @@
 // the next size is taken instead if it keeps more slice registers busy across the GPU (9 for 152 K).
 //
 //   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
-//             pieces counted on the stage's `full` barrier, never multicast); as soon as the
+//             pieces counted on the stage's `full` barrier, one destination CTA each); as soon as the
 //             consumers report a stage `done` it loads the row NS ahead into it.
 //   consumer  warp w owns a fixed slice of the segment and is independent of the other warps:
 //       front(i)  the slice is read from shared memory ONCE into registers (IT vectors per lane);
@@ -122,7 +122,7 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, uint32_t l
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-// Global -> this CTA's shared memory, completion counted on an mbarrier.  No multicast.
+// Global -> this CTA's shared memory, completion counted on an mbarrier; one destination CTA.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, void* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
