@@ -197,8 +197,8 @@ def test_whole_path_chained_on_its_own_outputs():
 
 # ---- rows large enough for the cluster-resident path (V >= 16384, V % 8 == 0, aligned) -----------
 
-@pytest.mark.parametrize("V,G,len_hi", [(16384, 6, 24),      # eight full segments; > 74 clusters' worth of rows
-                                        (20008, 2, 12),      # ragged last segment (2501 vectors over 8 CTAs)
+@pytest.mark.parametrize("V,G,len_hi", [(16384, 6, 24),      # one CTA per row; more rows than resident CTAs
+                                        (20008, 2, 12),      # two CTAs per row, ragged last segment (2501 vectors)
                                         (50000, 2, 10),
                                         (151936, 1, 8)])     # the Qwen vocabulary
 def test_cluster_path_vocab_sizes(V, G, len_hi):
