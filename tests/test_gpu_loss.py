@@ -270,6 +270,15 @@ def test_long_rows_up_to_and_beyond_the_cluster_path_limit(V):
     _check(b, _gpu_loss(b), oracle_loss(b))
 
 
+@pytest.mark.parametrize("V", [65536, 86016, 98304, 114688, 131072])       # four to eight CTAs per row
+def test_every_portable_cluster_size(V):
+    w = shrink(wl.WORKLOADS["c2_qwen_vocab"], V=V, G=1, n=8, m=4, len_lo=6, len_hi=12, seed=V % 101)
+    b = build_batch(w)
+    got = _gpu_loss(b)
+    _check(b, got, oracle_loss(b))
+    assert _gpu_loss(b, in_place=True)[2].tobytes() == got[2].tobytes()
+
+
 def test_long_rows_on_the_two_stage_ring_with_several_rows_per_cluster():
     """V = 327680 over 16 CTAs: segments of 40 KB, too long for three stages with two CTAs per SM, so the ring
     has two stages; 14 such clusters are resident at most, so with > 80 rows every stage is reused several times."""
