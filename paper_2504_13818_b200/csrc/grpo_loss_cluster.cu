@@ -185,11 +185,16 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
     const int nvec = a.V / 8;
     const int seg0 = (int)rank * seg_vecs;                                   // first vector of my segment
     const int cnt = max(0, min(seg_vecs, nvec - seg0));                      // vectors in my segment
-    const int stage_vecs = (seg_vecs + 7) & ~7;                              // stages start on 128-byte lines
+    const int stage_vecs = 32 * IT * kConsumerWarps;                         // a stage: IT whole blocks of 32 vectors per warp
     const int64_t n_rows = cluster_id < a.T ? (a.T - cluster_id + n_clusters - 1) / n_clusters : 0;
     const bool has_ref = a.ref_logp != nullptr && a.beta != 0.0f;
 
     if (tid < 2 * kSlots) (&c.xslot[0][0])[tid] = 0ull;            // tag 0 is no row's tag
+    // beyond the segment every stage holds -inf for good, so the sweeps load whole blocks without a bounds
+    // test: the copies and the write-back of the exponentials never reach there
+    for (int st = 0; st < n_stages; ++st)
+        for (int j = cnt + tid; j < stage_vecs; j += kThreads)
+            bufs[(size_t)st * stage_vecs + j] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&c.full[s], 1);                  // the copy issuer, with the byte count
@@ -365,9 +370,8 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
         }
     } else {
         // =================================== consumer warps ===================================
-        const int per_warp = ((cnt + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;     // slices start on 128-byte lines
-        const int lo = min(cnt, warp * per_warp), hi = min(cnt, lo + per_warp);    // my slice of the segment
-        const uint4 kNegInf4 = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+        // my slice of the stage: IT blocks of 32 vectors, of which those below hi belong to the segment
+        const int lo = warp * 32 * IT, hi = max(lo, min(cnt, lo + 32 * IT));
 
         // back(i): the gradient of row i over my slice, once the exchange warp has published its factors
         auto back = [&](int64_t i, int s) {
@@ -395,7 +399,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
 #pragma unroll
                 for (int k = 0; k < IT; ++k) {
                     const int j = lo + lane + 32 * k;
-                    q[k] = j < hi ? buf[j] : make_uint4(0u, 0u, 0u, 0u);
+                    q[k] = buf[j];
                 }
 #pragma unroll
                 for (int k = 0; k < IT; ++k) {
@@ -424,7 +428,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
 #pragma unroll
             for (int k = 0; k < IT; ++k) {
                 const int j = lo + lane + 32 * k;
-                q[k] = j < hi ? buf[j] : kNegInf4;
+                q[k] = buf[j];                                      // -inf beyond the segment
             }
             uint32_t pm[4] = {kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair};
 #pragma unroll
@@ -488,29 +492,33 @@ __global__ void bounded_wait_selftest_kernel(uint32_t polls, uint32_t* status) {
 constexpr size_t kHalfSmBytes = 233472 / 2 - 1024;      // what a CTA may hold for two of them to share an SM
 
 struct ClusterPlan {
-    int seg_vecs, n_stages;
+    int seg_vecs;        // vectors of a row per CTA
+    int it;              // vectors per lane of a consumer warp's slice: the kernel's IT
+    int n_stages;
     size_t smem;
 };
 
-// Ring depth and residency for a row of nvec vectors over `cl` CTAs: three stages (one row being
-// loaded, one in front(), one waiting for back()) and as many CTAs per SM as then fit; two stages
-// when three do not fit at all.
-bool plan_cluster(int nvec, int cl, ClusterPlan* p) {
-    const size_t limit = 232448;
+// Segments, slice depth and ring for a row of nvec vectors over `cl` CTAs.  A stage holds 32 * it vectors
+// per consumer warp (4 KB * it).  Three stages (one row being loaded, one in front(), one waiting for
+// back()) if two CTAs then still share an SM, else two stages with two CTAs per SM, which beat three
+// stages with one CTA per SM by 3 % (measured, V = 155648 .. 196608).  false: does not fit that way.
+bool plan_cluster(int nvec, int cl, int min_it, int max_it, ClusterPlan* p) {
     p->seg_vecs = ((nvec + cl - 1) / cl + 7) & ~7;                               // segments start on 128-byte lines of the row
-    const size_t seg_bytes = (size_t)((p->seg_vecs + 7) & ~7) * 16;               // a stage: the segment, padded to 128 bytes
-    if (seg_bytes >= (1u << 20)) return false;
+    const int block = 32 * kConsumerWarps;
+    p->it = (p->seg_vecs + block - 1) / block;
+    if (p->it < min_it) p->it = min_it;
+    if (p->it > max_it) return false;
+    const size_t stage_bytes = (size_t)p->it * block * 16;
     for (int stages = kMaxStages; stages >= 2; --stages) {
         p->n_stages = stages;
-        p->smem = (size_t)ctrl_bytes(cl) + (size_t)stages * seg_bytes;
-        if (p->smem <= limit) return true;
+        p->smem = (size_t)ctrl_bytes(cl) + (size_t)stages * stage_bytes;
+        if (p->smem <= kHalfSmBytes) return true;
     }
     return false;
 }
 
 template <int CL, int IT>
-int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t stream, bool* launched) {
-    ClusterPlan plan = plan_in;
+int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan, cudaStream_t stream, bool* launched) {
     auto kernel = grpo_loss_cluster_kernel<CL, IT>;
     PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem));
     if (CL > 8) PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
@@ -538,105 +546,27 @@ int launch_cluster_it(const RowArgs& a, const ClusterPlan& plan_in, cudaStream_t
     return PODS_OK;
 }
 
-// IT = vectors per lane of a consumer warp's slice.  Every depth a cluster size can be chosen with is
-// instantiated (unused lanes of the last vector cost as much as used ones, so rounding IT up to an even
-// number cost up to 15 % where it applied).  A size is only chosen when the size before it does not fit,
-// so its segments are at least that share of the largest one that fits and its depths start at kMinIt;
-// all sizes but the largest are bounded by the two-CTAs-per-SM segment (depth 10), the largest by the
-// register file (depth 12, with a ring of two stages, or one CTA per SM, for its longest segments).
-// A size may also be chosen in place of the previous one at depth 10 (see pick_cluster), which lowers
-// the first depth of sizes 3, 4 and 16 by one.
-template <int CL> constexpr int kMinIt = CL == 1 ? 1 : CL == 2 ? 5 : CL == 3 ? 6 : (CL == 4 || CL == 16) ? 7 : 8;
-template <int CL> constexpr int kMaxIt = CL == 16 ? 12 : 10;
-constexpr int kDeepestPairedIt = 10;          // the deepest slices whose segment still fits twice per SM
-
-// vectors per lane of a consumer warp's slice of a segment: slices start on 128-byte lines
-int slice_depth(int seg_vecs) {
-    const int per_warp = ((seg_vecs + kConsumerWarps - 1) / kConsumerWarps + 7) & ~7;
-    return (per_warp + 31) / 32;
-}
+// Slice depths each cluster size is instantiated for.  With the full ring and two CTAs per SM a stage holds
+// at most 9 blocks per warp (3 x 36 KB + control <= 113 KB), i.e. segments of up to 2304 vectors.  A size
+// is only chosen when the size before it does not fit, so its segments are at least that share of 2304
+// vectors and its depths start at kMinIt; the largest size goes on to depth 12 on a ring of two stages.
+template <int CL> constexpr int kMinIt = CL == 1 ? 1 : CL == 2 ? 5 : (CL == 3 || CL == 4 || CL == 16) ? 7 : CL <= 8 ? 8 : CL == 12 ? 8 : 9;
+template <int CL> constexpr int kMaxIt = CL == 16 ? 12 : 9;
 
 template <int CL, int IT>
-int launch_cluster_from(int it, const RowArgs& a, const ClusterPlan& plan, cudaStream_t stream, bool* launched) {
-    if (it <= IT) return launch_cluster_it<CL, IT>(a, plan, stream, launched);
-    if constexpr (IT < kMaxIt<CL>) return launch_cluster_from<CL, IT + 1>(it, a, plan, stream, launched);
-    return PODS_OK;                                                        // rows too long for the register-held slices
+int launch_cluster_from(const RowArgs& a, const ClusterPlan& plan, cudaStream_t stream, bool* launched) {
+    if (plan.it == IT) return launch_cluster_it<CL, IT>(a, plan, stream, launched);
+    if constexpr (IT < kMaxIt<CL>) return launch_cluster_from<CL, IT + 1>(a, plan, stream, launched);
+    return PODS_OK;
 }
 
+// Launches on clusters of CL if the row fits: with the full ring, or (any_ring) with the ring of two as well.
 template <int CL>
-int launch_cluster(const RowArgs& a, cudaStream_t stream, bool* launched) {
-    *launched = false;
+bool try_cluster(const RowArgs& a, bool any_ring, cudaStream_t stream, bool* launched, int* rc) {
     ClusterPlan plan;
-    if (!plan_cluster(a.V / 8, CL, &plan)) return PODS_OK;                 // does not fit: caller falls back
-    // segments too long for two CTAs per SM with the full ring: two CTAs with a ring of two beat one CTA
-    // with a ring of three (measured, V = 155648 .. 196608: +3 %)
-    const size_t seg_bytes = (size_t)((plan.seg_vecs + 7) & ~7) * 16;
-    if (plan.smem > kHalfSmBytes && ctrl_bytes(CL) + 2 * seg_bytes <= kHalfSmBytes) {
-        plan.n_stages = 2;
-        plan.smem = ctrl_bytes(CL) + 2 * seg_bytes;
-    }
-    return launch_cluster_from<CL, kMinIt<CL>>(slice_depth(plan.seg_vecs), a, plan, stream, launched);
-}
-
-// CTAs of this kernel that are resident at once when launched as clusters of CL with two CTAs per SM
-// (cluster placement leaves some of the 2 x SMs slots empty, how many depends on CL); -1 if the query fails.
-// Asked once per device.
-template <int CL>
-int resident_ctas() {
-    static int cached[64];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-    int v = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED);
-    if (v != 0) return v;
-    auto kernel = grpo_loss_cluster_kernel<CL, kDeepestPairedIt>;
-    v = -1;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CL;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3(CL, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kHalfSmBytes;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHalfSmBytes) == cudaSuccess &&
-        (CL <= 8 || cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) &&
-        cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0)
-        v = n * CL;
-    else
-        (void)cudaGetLastError();
-    __atomic_store_n(&cached[dev], v, __ATOMIC_RELAXED);
-    return v;
-}
-
-// Launches on clusters of CL if the row's segments fit the full ring twice per SM; false if they do not.
-// At the deepest slices (depth 10) the next size NEXT takes over when it promises more: resident CTAs
-// x the share of the slice registers that hold data.  Measured, 2 GiB of logits: V = 129280 and 131072
-// 8 CTAs per row instead of 7 +3 %, 151936 and 152064 9 instead of 8 +2 %; at lower depths the same
-// product picked the slower size more often than not (40960, 49152, 86016, 100352), so there the smaller
-// size stays.
-template <int CL, int NEXT>
-bool pick_cluster(const RowArgs& a, cudaStream_t stream, bool* launched, int* rc) {
-    const int nvec = a.V / 8;
-    ClusterPlan p;
-    if (!(plan_cluster(nvec, CL, &p) && p.n_stages == kMaxStages && p.smem <= kHalfSmBytes)) return false;
-    if constexpr (NEXT != 0) {
-        ClusterPlan q;
-        if (slice_depth(p.seg_vecs) == kDeepestPairedIt && plan_cluster(nvec, NEXT, &q) && q.n_stages == kMaxStages &&
-            q.smem <= kHalfSmBytes) {
-            const int dq = slice_depth(q.seg_vecs) < kMinIt<NEXT> ? kMinIt<NEXT> : slice_depth(q.seg_vecs);
-            const double here = (double)resident_ctas<CL>() * nvec / ((double)CL * kDeepestPairedIt);
-            const double next = (double)resident_ctas<NEXT>() * nvec / ((double)NEXT * dq);
-            if (here > 0.0 && next > here) {
-                *rc = launch_cluster<NEXT>(a, stream, launched);
-                if (*rc != PODS_OK || *launched) return true;
-            }
-        }
-    }
-    *rc = launch_cluster<CL>(a, stream, launched);
+    if (!plan_cluster(a.V / 8, CL, kMinIt<CL>, kMaxIt<CL>, &plan)) return false;
+    if (plan.n_stages < kMaxStages && !any_ring) return false;
+    *rc = launch_cluster_from<CL, kMinIt<CL>>(a, plan, stream, launched);
     return true;
 }
 
@@ -668,17 +598,18 @@ int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launch
     *launched = false;
     if (!a.vec_ok || a.V % 8 != 0 || a.V < __atomic_load_n(&g_cluster_min_vocab, __ATOMIC_RELAXED)) return PODS_OK;
     // as few CTAs per row as leave room for the full ring with two CTAs per SM: fewer partners to exchange
-    // with, longer slices per warp, and small clusters fill the GPU better than large ones; 11 and 13 to 15
-    // place badly (231 and at most 221 of the 296 CTA slots of a B200)
+    // with, and small clusters fill the GPU better than large ones (resident CTAs of the 296 slots of a B200,
+    // from cudaOccupancyMaxActiveClusters: sizes 1, 2: 296; 3: 279; 4: 284; 5: 280; 6: 270; 7: 259; 8: 264;
+    // 9: 270; 10: 260; 11: 231; 12: 252; 13: 221; 14: 196; 15: 210; 16: 224 - hence no 11 and no 13 to 15)
     int rc = PODS_OK;
-    if (pick_cluster<1, 2>(a, stream, launched, &rc) || pick_cluster<2, 3>(a, stream, launched, &rc) ||
-        pick_cluster<3, 4>(a, stream, launched, &rc) || pick_cluster<4, 5>(a, stream, launched, &rc) ||
-        pick_cluster<5, 6>(a, stream, launched, &rc) || pick_cluster<6, 7>(a, stream, launched, &rc) ||
-        pick_cluster<7, 8>(a, stream, launched, &rc) || pick_cluster<8, 9>(a, stream, launched, &rc) ||
-        pick_cluster<9, 10>(a, stream, launched, &rc) || pick_cluster<10, 12>(a, stream, launched, &rc) ||
-        pick_cluster<12, 16>(a, stream, launched, &rc))
+    if (try_cluster<1>(a, false, stream, launched, &rc) || try_cluster<2>(a, false, stream, launched, &rc) ||
+        try_cluster<3>(a, false, stream, launched, &rc) || try_cluster<4>(a, false, stream, launched, &rc) ||
+        try_cluster<5>(a, false, stream, launched, &rc) || try_cluster<6>(a, false, stream, launched, &rc) ||
+        try_cluster<7>(a, false, stream, launched, &rc) || try_cluster<8>(a, false, stream, launched, &rc) ||
+        try_cluster<9>(a, false, stream, launched, &rc) || try_cluster<10>(a, false, stream, launched, &rc) ||
+        try_cluster<12>(a, false, stream, launched, &rc) || try_cluster<16>(a, true, stream, launched, &rc))
         return rc;
-    return launch_cluster<16>(a, stream, launched);
+    return PODS_OK;                                       // rows too long for the register-held slices
 }
 
 }  // namespace pods_loss

@@ -261,7 +261,8 @@ def test_cluster_path_without_reference_policy_and_single_rows():
                                180224,      # ten
                                196608,      # twelve
                                262144,      # sixteen
-                               301056,      # sixteen, the longest segment with three stages and two CTAs per SM
+                               294912,      # sixteen, the longest segment with three stages and two CTAs per SM
+                               294920,      # one vector more: the ring of two stages
                                393216,      # sixteen, twelve vectors per lane: the deepest register-held slice
                                393224])     # one vector more: back to the general row kernel
 def test_long_rows_up_to_and_beyond_the_cluster_path_limit(V):
