@@ -33,7 +33,7 @@ from paper_2504_13818_b200 import workloads as wl  # noqa: E402
 METRIC = "kept-token GRPO loss+grad tokens/s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-NCU_DRAM_BYTES_PER_ROW = 598049      # ncu capture of grpo_loss_cluster_kernel at V = 151936, see profiles/
+NCU_DRAM_BYTES_PER_ROW = 597643      # ncu capture of grpo_loss_cluster_kernel at V = 151936, see profiles/
 
 
 def parse_args():
@@ -328,7 +328,7 @@ def run_ours(args):
     roofline = {"kernel": "grpo_loss_cluster_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
                 "frac_of_nominal_8TBps": achieved / 8000.0,
-                # dram__bytes_read.sum + dram__bytes_write.sum per launch: 598,049 B per row measured on the 4668-row
+                # dram__bytes_read.sum + dram__bytes_write.sum per launch: 597,643 B per row measured on the 4668-row
                 # capture of this kernel (profiles/), scaled to this launch's rows (traffic is proportional to rows)
                 "traffic": NCU_DRAM_BYTES_PER_ROW * batch.chunk if w.V == 151936 else None,
                 "bytes_per_launch": bytes_per_token * batch.chunk, "ms_per_launch": per_launch_ms,
