@@ -32,7 +32,7 @@ def _rank_main(rank, world, port, out):
 
 def test_two_ranks_report_the_slowest_time_and_the_summed_rate():
     world, port = 2, _free_port()
-    with mp.Manager() as manager:
+    with mp.get_context("spawn").Manager() as manager:
         out = manager.dict()
         mp.spawn(_rank_main, args=(world, port, out), nprocs=world, join=True)
         got = dict(out)
