@@ -412,12 +412,13 @@ def test_flat_rows_and_wide_logit_ranges(V):
 
 
 def test_repeated_launches_are_bit_identical_on_every_kernel_in_and_out_of_place():
-    """A few hundred launches per shape (row-tile kernel, row kernel, clusters of 1, 3 and 8 CTAs): any race in
-    the pipelines or the exchange would show as a differing bit or a status bit sooner or later."""
+    """A few hundred launches per shape (row-tile kernel, row kernel, clusters of 1, 3, 9 and 16 CTAs, the last on
+    the ring of two stages): any race in the pipelines or the exchange would show as a differing bit or a status
+    bit sooner or later."""
     dev = torch.device("cuda")
     g = torch.Generator(device=dev)
     g.manual_seed(11)
-    for V, T in [(1024, 700), (6000, 300), (12288, 900), (40960, 500), (151936, 150)]:
+    for V, T in [(1024, 700), (6000, 300), (12288, 900), (40960, 500), (151936, 150), (327680, 60)]:
         logits = (torch.randn((T, V), generator=g, device=dev) * 3).to(torch.bfloat16)
         tokens = torch.randint(0, V, (T,), generator=g, device=dev, dtype=torch.int32)
         cu = torch.linspace(0, T, 9, device=dev).long()
