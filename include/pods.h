@@ -6,10 +6,10 @@
  *
  * Conventions for every call
  *   - Pointers marked [dev] are device pointers on the current CUDA device, [host] are host
- *     pointers.  The caller owns every buffer; the library allocates no device memory and
- *     keeps no state between calls (except pods_host_step_*, which says what it allocates,
- *     grpo_loss_chunk_static, which says what it holds, and one tuning value, see
- *     pods_set_loss_cluster_min_vocab).
+ *     pointers.  The caller owns every buffer.  Three things outlive a call and are described
+ *     where they are declared: the object pods_host_step_create allocates, the fixed scratch
+ *     array grpo_loss_chunk_static uses, and the process-wide tuning value of
+ *     pods_set_loss_cluster_min_vocab.  No other call allocates device memory or keeps state.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
  *     enqueue work and return; outputs are valid once the stream has reached that point.
  *   - The return value is a pods_status.  Errors that the host can see (sizes, null or
@@ -90,8 +90,8 @@ int pods_select(const float* rewards, int64_t G, int32_t n, int32_t m, int32_t r
                 uint32_t flags, int32_t* idx, float* adv, int32_t* k_out, uint32_t* status, void* stream);
 
 /*
- * pods_compact - "apply the same procedure to each prompt and then concatenate the down-sampled
- * rollouts" (text after Algorithm 1).  Rollout j of group g is row g*n+j of the padded storage;
+ * pods_compact - concatenation of the kept rollouts of all prompt groups into one packed batch
+ * (text after Algorithm 1).  Rollout j of group g is row g*n+j of the padded storage;
  * kept rollout number i = g*m+j' is rollout idx[g,j'].
  *
  *   idx        [dev] int32 [G,m]                   lengths   [dev] int32 [G*n] tokens per rollout

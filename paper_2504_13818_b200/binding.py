@@ -95,6 +95,30 @@ def _dev(t, dtype, name, optional=False):
     return C.c_void_p(t.data_ptr())
 
 
+def _require(cond, message):
+    if not cond:
+        raise PodsError(message)
+
+
+def _numel(t, count, name):
+    """The C ABI sees pointers only: a short buffer would be read or written past its end on the device,
+    so every length is checked here, before the call."""
+    _require(t is None or t.numel() == count, "%s must hold %d entries, got %d" % (name, count, 0 if t is None else t.numel()))
+
+
+def _check_loss_shapes(logits, dlogits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, mask, logp):
+    _require(isinstance(logits, torch.Tensor) and logits.dim() == 2, "logits must be [T,V]")
+    T = logits.shape[0]
+    _require(tuple(dlogits.shape) == tuple(logits.shape), "dlogits must have the shape of logits %s, got %s"
+             % (tuple(logits.shape), tuple(dlogits.shape)))
+    M = cu_seqlens.numel() - 1
+    _require(M >= 1, "cu_seqlens must hold M+1 >= 2 entries")
+    for t, name in ((tokens, "tokens"), (old_logp, "old_logp"), (ref_logp, "ref_logp"), (mask, "mask"), (logp, "logp")):
+        _numel(t, T, name)
+    _numel(adv, M, "adv")
+    _numel(seq_weight, M, "seq_weight")
+
+
 def _rows(t, name):
     """Pointer and row pitch of a 2-D bf16 tensor whose rows are contiguous."""
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 2):
@@ -124,6 +148,7 @@ def pods_select(rewards, m, rule=RULE_MAXVAR, seed=0, flags=0, status=None, want
     if rewards.dim() != 2:
         raise PodsError("rewards must be [G,n]")
     G, n = rewards.shape
+    _require(1 <= m <= n, "need 1 <= m <= n, got m=%d n=%d" % (m, n))
     idx = torch.empty((G, m), dtype=torch.int32, device=rewards.device)
     adv = torch.empty((G, m), dtype=torch.float32, device=rewards.device)
     k = torch.empty((G,), dtype=torch.int32, device=rewards.device) if want_k else None
@@ -136,7 +161,12 @@ def pods_select(rewards, m, rule=RULE_MAXVAR, seed=0, flags=0, status=None, want
 
 def pods_select_into(rewards, m, idx, adv, k=None, rule=RULE_MAXVAR, seed=0, flags=0, status=None):
     """As pods_select with caller-provided outputs (no allocation)."""
+    _require(isinstance(rewards, torch.Tensor) and rewards.dim() == 2, "rewards must be [G,n]")
     G, n = rewards.shape
+    _require(1 <= m <= n, "need 1 <= m <= n, got m=%d n=%d" % (m, n))
+    _numel(idx, G * m, "idx")
+    _numel(adv, G * m, "adv")
+    _numel(k, G, "k")
     rc = load().pods_select(_dev(rewards, torch.float32, "rewards"), G, n, m, rule, seed, flags,
                             _dev(idx, torch.int32, "idx"), _dev(adv, torch.float32, "adv"),
                             _dev(k, torch.int32, "k", True), _dev(status, torch.int32, "status", True), _stream())
@@ -161,6 +191,15 @@ def pods_compact(idx, n, lengths, src_tokens, src_f32=(), T_cap=None, status=Non
         dst = [torch.empty(T_cap, dtype=torch.float32, device=dev) for _ in src_f32]
     else:
         cu, toks, dst = out
+    _require(idx.dim() == 2 and src_tokens.dim() == 2, "idx must be [G,m] and src_tokens [G*n, src_ld]")
+    _require(1 <= m <= n, "need 1 <= m <= n, got m=%d n=%d" % (m, n))
+    _numel(lengths, G * n, "lengths")
+    _require(src_tokens.shape[0] == G * n, "src_tokens must have G*n = %d rows, got %d" % (G * n, src_tokens.shape[0]))
+    _numel(cu, M + 1, "cu_seqlens")
+    _require(toks.numel() >= T_cap, "dst_tokens must hold T_cap = %d entries, got %d" % (T_cap, toks.numel()))
+    _require(len(dst) == len(src_f32), "one destination stream per source stream")
+    for d in dst:
+        _require(d.numel() >= T_cap, "dst_f32 streams must hold T_cap = %d entries, got %d" % (T_cap, d.numel()))
     k = len(src_f32)
     src_arr = (C.c_void_p * max(k, 1))(*[_dev(s, torch.float32, "src_f32").value for s in src_f32])
     dst_arr = (C.c_void_p * max(k, 1))(*[_dev(d, torch.float32, "dst_f32").value for d in dst])
@@ -180,6 +219,8 @@ def pods_compact(idx, n, lengths, src_tokens, src_f32=(), T_cap=None, status=Non
 def grpo_seq_weights(mask, cu_seqlens, out=None):
     M = cu_seqlens.shape[0] - 1
     w = out if out is not None else torch.empty(M, dtype=torch.float64, device=cu_seqlens.device)
+    _require(M >= 1, "cu_seqlens must hold M+1 >= 2 entries")
+    _numel(w, M, "seq_weight")
     rc = load().grpo_seq_weights(_dev(mask, torch.uint8, "mask", True), _dev(cu_seqlens, torch.int64, "cu_seqlens"),
                                  M, _dev(w, torch.float64, "seq_weight"), _stream())
     _check(rc, "grpo_seq_weights")
@@ -197,6 +238,8 @@ def grpo_loss_workspace_bytes(T, M, chunk_rows=0) -> int:
 def grpo_loss_chunk(logits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, row0, mask, eps, beta,
                     loss_acc, logp, dlogits, workspace, grad_scale=1.0, status=None):
     """One chunk of rows [row0, row0+T_chunk).  Per-token tensors hold this chunk's rows only."""
+    _check_loss_shapes(logits, dlogits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, mask, logp)
+    _numel(loss_acc, 1, "loss_acc")
     lp, ldl = _rows(logits, "logits")
     dp, ldd = _rows(dlogits, "dlogits")
     T, V = logits.shape
@@ -221,6 +264,8 @@ def grpo_loss_chunk_static(logits, tokens, old_logp, ref_logp, adv, seq_weight, 
 
     At most grpo_loss_chunk_static_max_rows() rows per call; calls on one device share the scratch, so
     they must not overlap on the GPU.  This wrapper itself creates no tensor."""
+    _check_loss_shapes(logits, dlogits, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, mask, logp)
+    _numel(loss_acc, 1, "loss_acc")
     lp, ldl = _rows(logits, "logits")
     dp, ldd = _rows(dlogits, "dlogits")
     T, V = logits.shape
@@ -270,6 +315,9 @@ def grpo_loss_fwd_bwd(logits, tokens, old_logp, ref_logp, adv, mask, eps, beta, 
     need = grpo_loss_workspace_bytes(T, M, chunk_rows)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    _check_loss_shapes(logits, dlogits, tokens, old_logp, ref_logp, adv, None, cu_seqlens, mask, logp)
+    _numel(loss, 1, "loss")
+    _require(workspace.numel() >= need, "workspace must hold %d bytes, got %d" % (need, workspace.numel()))
     lp, ldl = _rows(logits, "logits")
     dp, ldd = _rows(dlogits, "dlogits")
     rc = load().grpo_loss_fwd_bwd(lp, ldl, _dev(tokens, torch.int32, "tokens"), _dev(old_logp, torch.float32, "old_logp"),

@@ -193,6 +193,16 @@ grpo_loss_rows_kernel(const RowArgs a) {
 
         // ---- sweep 2: sum of exponentials, one instance of the maximum left out ---------------
         float s_t = 0.0f;
+        if (a.precise) {
+            // small chunk: e^(x - M) in fp64, no reference exponent and no correction factor
+            double sd = 0.0;
+            for (int v = tid; v < nvec; v += BLOCK) sd += exact_exp_sum(ld_global_v4(row4 + v), mx, v == excl);
+            for (int e = tail0 + tid; e < V; e += BLOCK) {
+                const float x = __uint_as_float((uint32_t)row[e] << 16);
+                if (nvec + (e - tail0) != excl && x != -INFINITY) sd += exp((double)x - (double)mx);
+            }
+            block_sum<BLOCK>(sd, sh);
+        } else {
         {
             uint4 nxt[kBatch];
             load_batch<BLOCK>(nxt, row4, tid, nvec);
@@ -213,12 +223,13 @@ grpo_loss_rows_kernel(const RowArgs a) {
             if (nvec + (e - tail0) != excl) s_t += ex2_approx(fmaf(x, kLog2e, -ref));
         }
         block_sum<BLOCK>((double)s_t, sh);
+        }
 
         // ---- scalar terms of the row (one thread, fp64) ---------------------------------------
         if (tid == 0) {
             const double corr = ref_correction(mx, ref);
             const RowInputs in = load_row_inputs(a, t);
-            const RowScalars r = row_scalars(a, in, x_tok, mx, sh.zprime * corr);
+            const RowScalars r = row_scalars(a, in, x_tok, mx, a.precise ? sh.zprime : sh.zprime * corr);
             a.logp[t] = (float)r.logp;
             a.row_loss[t] = r.weighted_loss;
             sh.coef = (float)(-r.g / r.Z * corr);
@@ -299,11 +310,12 @@ constexpr int kTileWarps = 8;
 constexpr int kTileMaxRows = 64;
 constexpr int kTileBytes = 64 * 1024;
 
-template <int IT>
+template <int IT, bool EXACT_SUM>
 __global__ void __launch_bounds__(kTileWarps * 32)
 grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
     extern __shared__ __align__(16) uint4 tile[];
     __shared__ float s_mx[kTileMaxRows], s_sum[kTileMaxRows], s_coef[kTileMaxRows], s_target[kTileMaxRows];
+    __shared__ double s_sum_exact[EXACT_SUM ? kTileMaxRows : 1];
     __shared__ int s_mode[kTileMaxRows], s_tok[kTileMaxRows];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nvec = a.V / 8;
@@ -336,6 +348,14 @@ grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
                 for (int k = IT - 1; k >= 0; --k)
                     if (vec_max(q[k]) == mx) excl = k;
             }
+            if (EXACT_SUM) {
+                double sd = 0.0;
+#pragma unroll
+                for (int k = 0; k < IT; ++k) sd += exact_exp_sum(q[k], mx, k == excl);
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) sd += __shfl_xor_sync(PODS_FULL_MASK, sd, d);
+                if (lane == 0) s_sum_exact[r] = sd;
+            }
             float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
             for (int k = 0; k < IT; ++k) {
@@ -361,7 +381,8 @@ grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
             const float mx = s_mx[tid];
             const double corr = ref_correction(mx, mx * kLog2e);
             const RowInputs in = load_row_inputs(a, t);
-            const RowScalars r = row_scalars(a, in, x_tok, mx, (double)s_sum[tid] * corr);
+            // the gradient rows scale the stored e = 2^(x log2e - ref): their factor keeps the correction either way
+            const RowScalars r = row_scalars(a, in, x_tok, mx, EXACT_SUM ? s_sum_exact[tid] : (double)s_sum[tid] * corr);
             a.logp[t] = (float)r.logp;
             a.row_loss[t] = r.weighted_loss;
             s_coef[tid] = (float)(-r.g / r.Z * corr);
@@ -400,19 +421,30 @@ grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
     }
 }
 
-template <int IT>
-int launch_tile(const RowArgs& a, cudaStream_t s) {
+template <int IT, bool EXACT_SUM>
+int launch_tile_as(const RowArgs& a, cudaStream_t s) {
     const int nvec = a.V / 8;
     int rows = kTileBytes / (nvec * 16);
     rows = rows > kTileMaxRows ? kTileMaxRows : rows & ~(kTileWarps - 1);
+    // a small chunk is spread over the whole GPU: fewer rows per tile, more tiles
+    if (EXACT_SUM) {
+        const int64_t spread = (a.T + pods_sm_count() - 1) / pods_sm_count();
+        const int want = (int)((spread + kTileWarps - 1) / kTileWarps * kTileWarps);
+        rows = want < rows ? want : rows;
+    }
     const size_t smem = (size_t)rows * nvec * 16;
-    auto kernel = grpo_loss_tile_kernel<IT>;
+    auto kernel = grpo_loss_tile_kernel<IT, EXACT_SUM>;
     PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t tiles = (a.T + rows - 1) / rows;
     const int64_t cap = (int64_t)pods_sm_count() * 3;
     kernel<<<(unsigned)(tiles < cap ? tiles : cap), kTileWarps * 32, smem, s>>>(a, rows);
     PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
     return PODS_OK;
+}
+
+template <int IT>
+int launch_tile(const RowArgs& a, cudaStream_t s) {
+    return a.precise ? launch_tile_as<IT, true>(a, s) : launch_tile_as<IT, false>(a, s);
 }
 
 // Short rows on the row-tile kernel; *launched says whether the shape was taken.
@@ -480,6 +512,7 @@ extern "C" int grpo_loss_chunk(const void* logits, int64_t ldl, const int32_t* t
     a.prep = reinterpret_cast<RowPrep*>(static_cast<unsigned char*>(workspace) + align_up((size_t)T_chunk * sizeof(double), 256));
     a.status = status;
     a.vec_ok = pods_aligned(logits, 16) && pods_aligned(dlogits, 16) && ldl % 8 == 0 && ldd % 8 == 0;
+    a.precise = T_chunk * (int64_t)V <= kExactSumMaxLogits;
 
     cudaStream_t s = pods_stream(stream);
     bool on_cluster_path = false;

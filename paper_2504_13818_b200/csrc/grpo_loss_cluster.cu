@@ -6,12 +6,12 @@
 // so HBM sees exactly one read and one write per element and every other access is to shared
 // memory.  A CTA is eight consumer warps, one producer warp and one exchange warp that meet only
 // through mbarriers, over a ring of NS segment buffers; no warp ever waits at a CTA-wide barrier.
-// CL is chosen per launch: the smallest of 1 .. 10, 12, 16 whose segment leaves room for the
-// ring with two CTAs per SM (8 for a 128 K vocabulary, 1 for 16 K, 16 for 256 K): small clusters have
-// fewer partners to wait for and leave fewer CTA slots of the GPU empty (cluster placement fills 296
-// slots with clusters of 1 or 2, 264 with 8, 224 with 16).  Sizes above 8 are non-portable cluster
-// sizes, which the launch asks for explicitly.  Where the smallest size needs the deepest register slices,
-// the next size is taken instead if it keeps more slice registers busy across the GPU (9 for 152 K).
+// CL is chosen per launch: the smallest of 1 .. 10, 12, 16 whose padded stage (whole blocks of 32
+// vectors per consumer warp) leaves room for the ring with two CTAs per SM (1 for a 16 K vocabulary,
+// 8 for 128 K, 9 for 152 K, 16 from 222 K up): small clusters have fewer partners to wait for and leave
+// fewer CTA slots of the GPU empty (cluster placement fills 296 slots with clusters of 1 or 2, 264 with
+// 8, 270 with 9, 224 with 16).  Sizes above 8 are non-portable cluster sizes, which the launch asks for
+// explicitly.
 //
 //   producer  one thread: bulk asynchronous copies global -> shared of the row's segment (8 KB
 //             pieces counted on the stage's `full` barrier, one destination CTA each); as soon as the
@@ -31,6 +31,8 @@
 //                        on the stage's `done` barrier.
 //             front(i) runs before back(i-1), so the exchange of row i-1 has a whole sweep to finish.
 //             Shared memory sees 8 bytes of traffic per element (2 in, 2 read, 2 written, 2 read).
+//             A stage is written through both proxies (bulk copies in, bf16(e) by ordinary stores), so a
+//             consumer fences the two before it reports the stage done.
 //   exchange  for every row: writes the CTA's eight (m_w, sum_w) pairs into the slots it owns in
 //             every peer's shared memory, each as ONE 64-bit word that carries the row's tag, so
 //             that no fence or barrier crosses the cluster: a reader polls its 8 CL slots until all
@@ -66,8 +68,9 @@ constexpr int kPieceVecs = 512;               // 16-byte vectors per bulk load (
 __host__ __device__ constexpr int slot_count(int cl) { return cl <= 8 ? 64 : 128; }
 // barriers, row scalars and exchange slots ahead of the buffers
 __host__ __device__ constexpr int ctrl_bytes(int cl) { return cl <= 8 ? 1408 : 2432; }
-constexpr uint32_t kSpinLimit = 1u << 24;     // polls of one barrier or slot before giving up (a fraction of a second)
-constexpr uint32_t kSuspendNs = 1000;         // upper bound on the time one poll may suspend the thread
+constexpr uint32_t kSpinLimit = 1u << 24;     // polls of one barrier or slot before giving up
+constexpr uint32_t kSuspendNs = 1000;         // upper bound on the time one poll may suspend the thread: a wait
+                                              // that never completes ends after at most 2^24 us = 17 s
 
 struct Pair {
     uint32_t key;                             // ordered bf16 slice maximum in the upper half
@@ -411,6 +414,9 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 if (tok_vec >= lo && tok_vec < hi && ((tok_vec - lo) & 31) == lane)
                     reinterpret_cast<uint16_t*>(out)[(int64_t)tok_vec * 8 + (token & 7)] = target_bits;
             }
+            // The stage holds bf16(e) written by these lanes with ordinary stores; the producer refills it with
+            // bulk copies, which go through the asynchronous proxy: order the two before handing it back.
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();                              // every lane has its values: the stage may be loaded again
             if (lane == 0) mbar_arrive(&c.done[s]);
         };

@@ -165,7 +165,30 @@ struct RowArgs {
     RowPrep* prep;         // workspace [T]: the rows' scalar inputs (cluster path)
     uint32_t* status;
     int vec_ok;            // 16-byte aligned rows: 128-bit path
+    int precise;           // small chunk: the sum of exponentials is also taken in fp64 (see exact_sum_threshold)
 };
+
+// Chunks of at most this many logits are bound by launch latency, not by bandwidth: there the row-tile and
+// the general row kernel also take the sum of exponentials in fp64 with the library exponential, so that the
+// log-probs carry fp64 accuracy and a loss that is a nearly cancelling sum of rollout terms (zero-sum
+// advantages) keeps its relative accuracy.  The gradient rows are the same either way.
+constexpr int64_t kExactSumMaxLogits = 1 << 20;
+
+// Sum over a vector's eight values of e^(x - mx) in fp64; `skip_first_max` leaves out the first value equal to mx.
+static __device__ __noinline__ double exact_exp_sum(uint4 q, float mx, bool skip_first_max) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    double s = 0.0;
+    bool skipped = !skip_first_max;
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t word = w[i >> 1];
+        const float v = (i & 1) ? bf16_hi(word) : bf16_lo(word);
+        const bool skip = !skipped && v == mx;
+        skipped |= skip;
+        if (!skip && v != -INFINITY) s += exp((double)v - (double)mx);
+    }
+    return s;
+}
 
 // Rollout of packed row r: the i with cu_seqlens[i] <= r < cu_seqlens[i+1].
 __device__ __forceinline__ int64_t find_rollout(const int64_t* cu, int64_t M, int64_t r) {

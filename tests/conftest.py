@@ -17,3 +17,16 @@ def _built_oracle():
     """The C oracle is compiled on demand (gcc); building the checker is not using it."""
     from oracle import build
     build.build()
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _parity_record():
+    """GPU parity tests append the maxima they achieved (not only pass/fail) to gpurun_out/parity_maxima.jsonl."""
+    import parity
+    out = os.path.join(ROOT, "gpurun_out")
+    try:
+        os.makedirs(out, exist_ok=True)
+        parity.RECORD_PATH = os.path.join(out, "parity_maxima.jsonl")
+    except OSError:
+        parity.RECORD_PATH = None
+    yield

@@ -62,3 +62,74 @@ def test_cluster_vocabulary_limit_is_a_process_wide_setting_with_a_floor():
     assert lib.pods_set_loss_cluster_min_vocab(5) == 100000       # values below 2048 are raised to 2048
     assert lib.pods_set_loss_cluster_min_vocab(default) == 2048
     assert lib.pods_set_loss_cluster_min_vocab(default) == default
+
+
+def test_binding_checks_every_buffer_length_before_the_call():
+    """The C ABI cannot see buffer sizes, so the binding does: a short or mis-shaped tensor is refused on
+    the host.  Host tensors are enough to show it - the length checks come before anything is marshalled,
+    so nothing can have been launched when they raise."""
+    import pytest
+    import torch
+    T, V, M = 12, 16, 3
+    bf = torch.zeros((T, V), dtype=torch.bfloat16)
+
+    def loss_args(**over):
+        a = dict(logits=bf, tokens=torch.zeros(T, dtype=torch.int32), old_logp=torch.zeros(T), ref_logp=torch.zeros(T),
+                 adv=torch.zeros(M), seq_weight=torch.zeros(M, dtype=torch.float64),
+                 cu_seqlens=torch.zeros(M + 1, dtype=torch.int64), row0=0, mask=torch.ones(T, dtype=torch.uint8),
+                 eps=0.2, beta=0.04, loss_acc=torch.zeros(1, dtype=torch.float64), logp=torch.zeros(T),
+                 dlogits=torch.zeros_like(bf))
+        a.update(over)
+        return a
+
+    wrong = {"dlogits": torch.zeros((T - 1, V), dtype=torch.bfloat16), "tokens": torch.zeros(T - 1, dtype=torch.int32),
+             "old_logp": torch.zeros(T + 1), "ref_logp": torch.zeros(1), "mask": torch.ones(T - 2, dtype=torch.uint8),
+             "logp": torch.zeros(T - 1), "adv": torch.zeros(M + 1), "seq_weight": torch.zeros(M - 1, dtype=torch.float64),
+             "cu_seqlens": torch.zeros(M, dtype=torch.int64), "loss_acc": torch.zeros(2, dtype=torch.float64)}
+    ws = torch.zeros(1 << 16, dtype=torch.uint8)
+    for name, bad in wrong.items():
+        with pytest.raises(binding.PodsError, match="must hold|must have the shape"):
+            binding.grpo_loss_chunk(workspace=ws, **loss_args(**{name: bad}))
+        with pytest.raises(binding.PodsError, match="must hold|must have the shape"):
+            binding.grpo_loss_chunk_static(**loss_args(**{name: bad}))
+    for name in ("dlogits", "tokens", "old_logp", "ref_logp", "mask", "logp", "adv", "cu_seqlens"):
+        a = loss_args(**{name: wrong[name]})
+        for drop in ("seq_weight", "row0", "loss_acc"):
+            a.pop(drop)
+        with pytest.raises(binding.PodsError, match="must hold|must have the shape"):
+            binding.grpo_loss_fwd_bwd(workspace=ws, loss=torch.zeros(1), **a)
+    a = loss_args()
+    for drop in ("seq_weight", "row0", "loss_acc"):
+        a.pop(drop)
+    with pytest.raises(binding.PodsError, match="workspace must hold"):
+        binding.grpo_loss_fwd_bwd(workspace=torch.zeros(8, dtype=torch.uint8), loss=torch.zeros(1), **a)
+    # with every length right the first complaint is that these are host tensors: the checks above all passed
+    with pytest.raises(binding.PodsError, match="CUDA"):
+        binding.grpo_loss_chunk(workspace=ws, **loss_args())
+
+    G, n, m, ld = 2, 4, 2, 8
+    idx = torch.zeros((G, m), dtype=torch.int32)
+    lengths, src = torch.zeros(G * n, dtype=torch.int32), torch.zeros((G * n, ld), dtype=torch.int32)
+    good = (torch.zeros(G * m + 1, dtype=torch.int64), torch.zeros(G * m * ld, dtype=torch.int32), [])
+    with pytest.raises(binding.PodsError, match="lengths must hold"):
+        binding.pods_compact(idx, n, lengths[:-1], src, out=good)
+    with pytest.raises(binding.PodsError, match="rows"):
+        binding.pods_compact(idx, n, lengths, src[:-1], out=good)
+    with pytest.raises(binding.PodsError, match="cu_seqlens must hold"):
+        binding.pods_compact(idx, n, lengths, src, out=(good[0][:-1], good[1], []))
+    with pytest.raises(binding.PodsError, match="dst_tokens must hold"):
+        binding.pods_compact(idx, n, lengths, src, out=(good[0], good[1][:-1], []))
+    with pytest.raises(binding.PodsError, match="dst_f32 streams must hold"):
+        binding.pods_compact(idx, n, lengths, src, src_f32=[torch.zeros((G * n, ld))],
+                             out=(good[0], good[1], [torch.zeros(3)]))
+    r = torch.zeros((G, n))
+    with pytest.raises(binding.PodsError, match="idx must hold"):
+        binding.pods_select_into(r, m, torch.zeros((G, m + 1), dtype=torch.int32), torch.zeros((G, m)))
+    with pytest.raises(binding.PodsError, match="adv must hold"):
+        binding.pods_select_into(r, m, idx, torch.zeros((G, m - 1)))
+    with pytest.raises(binding.PodsError, match="k must hold"):
+        binding.pods_select_into(r, m, idx, torch.zeros((G, m)), torch.zeros(G + 1, dtype=torch.int32))
+    with pytest.raises(binding.PodsError, match="1 <= m <= n"):
+        binding.pods_select_into(r, n + 1, idx, torch.zeros((G, m)))
+    with pytest.raises(binding.PodsError, match="seq_weight must hold"):
+        binding.grpo_seq_weights(None, torch.zeros(M + 1, dtype=torch.int64), out=torch.zeros(M + 2, dtype=torch.float64))

@@ -1,9 +1,8 @@
 """The loss path at the full sizes of configs 2 and 5, in the launch configuration bench.py times
 (grpo_loss_chunk over 16384-row chunks at V = 151936), against the oracle:
 
-  * config 2 (36,853 kept tokens, 11.2 GB of logits): every row's log-prob and the loss against the
-    oracle over ALL rows; dlogits element by element on a sample of rows spread over every chunk and
-    every rollout boundary the sample happens to hit;
+  * config 2 (36,853 kept tokens, 11.2 GB of logits): every row's log-prob, the loss and every element of
+    dlogits against the oracle over ALL rows (the oracle runs in 1024-row blocks of fp64 gradient rows);
   * config 5 (about 2 x 10^5 kept tokens, 61 GB of logits, processed chunk by chunk in place): the first,
     a middle and the last chunk (they hold rollouts that straddle chunk edges): per chunk, every row's
     log-prob and the chunk's contribution to the loss against the oracle over the whole chunk, dlogits
@@ -17,7 +16,8 @@ import torch
 
 import oracle
 from paper_2504_13818_b200 import binding, workloads as wl
-from parity import CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, LOSS_COND, LOSS_RTOL, dlogits_ulp_error, gradient_slack
+from parity import (CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, LOSS_COND, LOSS_RTOL, assert_dlogits_close, dlogits_report,
+                    gradient_slack, record)
 
 pytestmark = pytest.mark.gpu
 
@@ -54,9 +54,18 @@ def _check_rows(b, rows, gpu_logp_rows, gpu_dl_bits):
     assert int(fragile.sum()) == 0
     slack = gradient_slack({"w": b["w"], "mask": b["mask"], "cu": b["cu"], "seq_of_row": b["seq_of_row"],
                             "adv32": b["adv32"], "old": b["old"], "ref": b["ref"]}, want, rows=rows)
-    worst = dlogits_ulp_error(gpu_dl_bits, want["dlogits"], slack).max()
-    assert worst <= DLOGITS_ULPS, "dlogits off by %.2f bf16 ulps" % worst
+    rep = dlogits_report(gpu_dl_bits, want["dlogits"], slack)
+    assert_dlogits_close(rep)
+    rep["logp_abs"] = float(np.abs(gpu_logp_rows - want["logp"]).max())
+    want["report"] = rep
     return want
+
+
+def _merge(total, rep):
+    for k in ("literal_ulps", "allowance_ulps", "logp_abs"):
+        total[k] = max(total.get(k, 0.0), rep[k])
+    for k in ("allowance_rows", "rows"):
+        total[k] = total.get(k, 0) + rep[k]
 
 
 @needs_big_gpu
@@ -93,29 +102,30 @@ def test_config2_at_bench_size_and_launch_configuration():
     assert binding.read_status(status) == 0
     np.testing.assert_allclose(sw_d.cpu().numpy(), sw, rtol=1e-15)
 
-    # oracle over all rows (log-probs, loss), in blocks so that the host copy of the logits stays small
+    # oracle over ALL rows: log-probs, loss terms and every gradient element, in blocks so that the fp64
+    # gradient rows of a block (1024 x 151936 x 8 B = 1.2 GB) stay small on the host
     ell = np.empty(T, np.float64)
     logp_o = np.empty(T, np.float64)
-    for lo in range(0, T, 4096):
-        hi = min(T, lo + 4096)
-        out = oracle.grpo_rows(logits[lo:hi].view(torch.uint16).cpu().numpy(), tokens[lo:hi], old[lo:hi], ref[lo:hi],
-                               adv32, sw, seq_of_row[lo:hi], mask[lo:hi], w.eps, w.beta, want_dlogits=False)
-        ell[lo:hi], logp_o[lo:hi] = out["ell"], out["logp"]
-    assert np.abs(logp.cpu().numpy() - logp_o).max() <= LOGP_ATOL
-    loss_o = oracle.grpo_loss(ell, mask, cu)
-    scale = np.mean([abs(ell[cu[i]:cu[i + 1]].mean()) for i in range(len(cu) - 1)])
-    assert abs(float(loss.item()) - loss_o) <= LOSS_RTOL * max(abs(loss_o), scale / LOSS_COND)
-    assert abs(float(loss.item()) - loss_o) <= LOSS_RTOL * abs(loss_o)       # this batch meets the literal bound too
-
-    # gradient rows, element by element, on a sample from every chunk
-    rng = np.random.default_rng(0)
     b = {"w": w, "tokens": tokens, "old": old, "ref": ref, "adv32": adv32, "sw": sw, "seq_of_row": seq_of_row,
          "mask": mask, "cu": cu}
-    for lo in range(0, T, chunk):
-        rows = _sample_rows(lo, min(T, lo + chunk), cu, 40, rng)
-        rows_d = torch.from_numpy(rows).to(dev)
-        b["logits_rows"] = logits[rows_d].view(torch.uint16).cpu().numpy()
-        _check_rows(b, rows, logp[rows_d].cpu().numpy(), dl[rows_d].view(torch.uint16).cpu().numpy())
+    total = {}
+    block = 1024
+    for lo in range(0, T, block):
+        hi = min(T, lo + block)
+        rows = np.arange(lo, hi, dtype=np.int64)
+        b["logits_rows"] = logits[lo:hi].view(torch.uint16).cpu().numpy()
+        out = _check_rows(b, rows, logp[lo:hi].cpu().numpy(), dl[lo:hi].view(torch.uint16).cpu().numpy())
+        ell[lo:hi], logp_o[lo:hi] = out["ell"], out["logp"]
+        _merge(total, out["report"])
+        del out
+    assert total["rows"] == T
+    loss_o = oracle.grpo_loss(ell, mask, cu)
+    scale = np.mean([abs(ell[cu[i]:cu[i + 1]].mean()) for i in range(len(cu) - 1)])
+    d = abs(float(loss.item()) - loss_o)
+    record("c2_qwen_vocab, all %d rows, 16384-row chunk launches" % T, V=w.V, loss=loss_o,
+           loss_rel_literal=d / abs(loss_o), loss_rel_conditioned=d / max(abs(loss_o), scale / LOSS_COND), **total)
+    assert d <= LOSS_RTOL * max(abs(loss_o), scale / LOSS_COND)
+    assert d <= LOSS_RTOL * abs(loss_o)       # this batch meets the literal bound too
 
 
 @needs_big_gpu
@@ -178,7 +188,11 @@ def test_config5_chunked_in_place_first_middle_and_last_chunk():
         full_old[lo:hi], full_ref[lo:hi] = old, ref
         b = {"w": w, "tokens": tokens, "old": full_old, "ref": full_ref, "adv32": adv32, "sw": sw,
              "seq_of_row": seq_of_row, "mask": mask, "cu": cu, "logits_rows": keep}
-        _check_rows(b, rows, logp[rows_d].cpu().numpy(), logits[rows_d].view(torch.uint16).cpu().numpy())
+        rep = _check_rows(b, rows, logp[rows_d].cpu().numpy(), logits[rows_d].view(torch.uint16).cpu().numpy())["report"]
+        record("c5_large_loss, chunk %d of %d in place" % (c, n_chunks), V=w.V, rows_logp=hi - lo,
+               logp_abs_all_rows=float(np.abs(logp.cpu().numpy() - out["logp"]).max()), chunk_loss_share=share_o,
+               share_rel_literal=abs(share - share_o) / abs(share_o),
+               share_rel_conditioned=abs(share - share_o) / max(abs(share_o), size / LOSS_COND), **rep)
         del host_bits
     assert straddling >= 2                                   # the checked chunks did cut rollouts in two
     assert binding.read_status(status) == 0 and np.isfinite(float(acc.item()))

@@ -4,14 +4,17 @@ Bar: per-token log-prob abs <= 1e-3, loss rel <= 1e-4 (see parity.assert_loss_cl
 cancel), dlogits within 2 bf16 ulps.  Rows whose
 min(rho a, clip(rho) a) is within CLIP_MARGIN of switching branch are compared on logp only (the
 branch is a floating-point decision; none is expected with these inputs and the count is asserted)."""
+import os
+
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2504_13818_b200 import binding, workloads as wl
-from parity import (CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, assert_loss_close, build_batch, dlogits_ulp_error,
-                    gradient_slack, oracle_loss, shrink)
+from parity import (CLIP_MARGIN, DLOGITS_ULPS, LOGP_ATOL, LOSS_RTOL, assert_dlogits_close, assert_loss_close,
+                    build_batch, dlogits_report, dlogits_ulp_error, gradient_slack, loss_errors, oracle_loss, record,
+                    shrink)
 
 pytestmark = pytest.mark.gpu
 
@@ -45,22 +48,31 @@ def _gpu_loss(b, chunk_rows=0, in_place=False, ref=True, beta=None, mask=None):
             binding.read_status(status))
 
 
-def _check(b, got, want, expect_fragile=0):
+def _check(b, got, want, expect_fragile=0, case=None, literal_loss=False):
+    """Log-probs, loss and gradient against the oracle.  Gradient rows whose factor g_t is not a cancellation
+    (all but a handful) are held to the literal 2-ulp bound; the count of the others is part of the record."""
     loss, logp, dl_bits, status = got
     assert status == 0
-    assert np.abs(logp - want["logp"]).max() <= LOGP_ATOL
-    assert_loss_close(loss, want, b)
+    logp_err = float(np.abs(logp - want["logp"]).max())
+    assert logp_err <= LOGP_ATOL
+    errs = loss_errors(loss, want, b)
     fragile = (want["margin"] < CLIP_MARGIN) & (want["margin"] > 0)
     assert int(fragile.sum()) == expect_fragile
-    ulps = dlogits_ulp_error(dl_bits, want["dlogits"], gradient_slack(b, want))
-    worst = ulps[~fragile].max() if (~fragile).any() else 0.0
-    assert worst <= DLOGITS_ULPS, "dlogits off by %.2f bf16 ulps" % worst
-    return worst
+    rep = dlogits_report(dl_bits, want["dlogits"], gradient_slack(b, want), skip_rows=fragile)
+    case = case or os.environ.get("PYTEST_CURRENT_TEST", "?").split("::", 1)[-1].replace(" (call)", "")
+    record(case, V=int(b["logits"].shape[1]), logp_abs=logp_err, **errs, **rep)
+    assert_loss_close(loss, want, b)
+    if literal_loss:
+        assert errs["loss_rel_literal"] <= LOSS_RTOL, errs
+    assert_dlogits_close(rep)
+    return rep["literal_ulps"]
 
 
-def test_config1_whole_path_values():
+def test_config1_whole_path_values(request):
+    """Config 1 in full.  Its loss is a nearly cancelling sum (rollout terms of +-0.06 add up to 1.7e-6): the
+    chunk is small enough for the exact fp64 sums, so the literal relative bound holds as well."""
     b = build_batch(wl.WORKLOADS["c1_tiny"])
-    _check(b, _gpu_loss(b), oracle_loss(b))
+    _check(b, _gpu_loss(b), oracle_loss(b), case="c1_tiny [%s]" % request.node.callspec.id, literal_loss=True)
 
 
 @pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 1000, 1024, 8200, 40001])
