@@ -4,12 +4,14 @@ Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
 package; the product (the CUDA library and its binding) never does, and this
 package imports nothing from the product.
 
-Three layers:
+Four parts:
   * ``definition``  - the selection rule as the paper defines it (maximise the
     variance over every m-subset), exact rational arithmetic, tiny inputs only;
   * ``pods_oracle.c`` (wrapped here) - Algorithm 2, the advantages and the
     GRPO-PODS objective with its gradient, fp64, any size;
-  * ``compact`` - concatenation of the kept rollouts (text after Algorithm 1).
+  * ``compact`` - concatenation of the kept rollouts (text after Algorithm 1);
+  * ``lm_head`` - the token log-probability when the logits are the projection hidden W^T
+    (pi_theta of Sections 3.1 / 3.2), fp64.
 """
 import ctypes as C
 import os
@@ -168,3 +170,4 @@ def grpo_loss(ell, mask, cu_seqlens):
 
 from .definition import max_variance_subsets, variance_exact  # noqa: E402,F401
 from .compact import compact  # noqa: E402,F401
+from . import lm_head  # noqa: E402,F401
