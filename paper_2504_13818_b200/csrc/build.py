@@ -25,12 +25,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = [f for f in NVCC_FLAGS if f not in ("--use_fast_math=false", "-shared")]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    # one nvcc per source, side by side (the sources share no device symbols), then one link
+    objdir = os.path.join(PKG, "_build")
+    os.makedirs(objdir, exist_ok=True)
+    jobs = []
+    for src in SOURCES:
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        jobs.append((obj, subprocess.Popen([nvcc] + flags + ["-c", src, "-o", obj])))
+    failed = [obj for obj, p in jobs if p.wait() != 0]
+    if failed:
+        raise subprocess.CalledProcessError(1, "nvcc -c (%s)" % ", ".join(os.path.basename(f) for f in failed))
     tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + flags + SOURCES + ["-o", tmp]
-    subprocess.run(cmd, check=True)
+    subprocess.run([nvcc, "-shared", "-Xcompiler", "-fPIC"] + [obj for obj, _ in jobs] + ["-o", tmp], check=True)
     os.replace(tmp, LIB)
     return LIB
 

@@ -1,18 +1,20 @@
 // pods_select: the down-sampling rule D(o, r; m) -> S (Definition 3.1) for G prompt groups per
 // launch, and the advantages of the kept subset (Section 3.2).
 //
+// Two kernels.  The max-variance and max-reward rules (Algorithm 2; the m highest) run on
+// pods_select_fast_kernel, described above its definition: a network sort of bare 32-bit keys, the
+// running sums and split scores of Theorem 1's proof in registers, and the kept set read off two
+// thresholds.  The random and percentile rules need every element's sorted position and run on
+// pods_select_kernel:
+//
 // One group is handled by LANES consecutive lanes of a warp (8, 16 or 32), each lane holding E
 // elements in registers (LANES * E >= n, padded with +infinity keys).  Steps, per group:
-//   1. load the rewards (coalesced), build a 64-bit key (order-preserving reward bits : index)
-//      so that one unsigned compare gives the stable (reward, index) order of argsort;
+//   1. load the rewards (coalesced), build a 64-bit key (order-preserving reward bits or the
+//      rollout's Philox word : index) so that one unsigned compare gives the stable order of argsort;
 //   2. bitonic sort: strides below E are compare-exchanges between registers of a lane, larger
-//      strides exchange with another lane by shuffle (Algorithm 2, step 1);
-//   3. fp64 running sums of the centred rewards and their squares over the sorted order, upward
-//      from the lowest and downward from the highest, written to shared memory (the prefix sums
-//      of Theorem 1's proof);
-//   4. each lane scores its share of the m+1 splits "k highest + (m-k) lowest" from the prefix
-//      sums, then a shuffle arg-max picks the largest score, smallest k (Algorithm 2, steps 2-6);
-//   5. kept elements are marked in a bitmap indexed by original index, then written out in
+//      strides exchange with another lane by shuffle;
+//   3. fp64 sums of the centred rewards over the kept subset (and the full group);
+//   4. kept elements are marked in a bitmap indexed by original index, then written out in
 //      ascending original index with a ballot compaction, together with their advantages.
 
 #include <math.h>
@@ -313,34 +315,88 @@ pods_select_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, i
 // v_hi - exactly the set the stable (reward, index) order picks.  So the network sorts bare 32-bit
 // keys (one min and one max per compare-exchange, no payload), in the form whose first step of
 // every merge level mirrors the block (position p against p ^ (k-1)) so that all steps put the
-// minimum at the lower position and no direction has to be selected.  A second sweep over the
-// rewards in original order (kept in registers) then emits indices and advantages.
+// minimum at the lower position and no direction has to be selected.
+//
+// A group is LANES lanes x E register elements.  Registers hold the keys only while they are being
+// sorted; the group's keys in original order and in sorted order live in shared memory (rows of E
+// words per lane, padded by four words so that 128-bit accesses of a quarter warp fall on distinct
+// banks), which lets every later phase pick the distribution of work it needs:
+//   sums     Algorithm 2 reads only the m lowest and the m highest sorted positions.  Those 2m values
+//            are dealt out evenly, c = ceil(m / LANES) consecutive positions of each end per lane;
+//            a lane sums its own, one scan over the group gives what lies below (lowest end) and
+//            from it upward (highest end), and the lane then walks its c splits with both running
+//            sums in registers: the split "j lowest + (m-j) highest" is scored by the lane that
+//            holds sorted position j, no value goes through memory;
+//   arg-max  three warp reductions on the order-preserving integer image of the fp64 score
+//            (high word, low word, then the largest j, i.e. the smallest k, among equal scores);
+//   classify every lane looks at its E rewards in original order and builds four bit masks
+//            (below v_lo, equal to it, above v_hi, equal to it); one packed scan over the group
+//            turns the counts into the number of ties to keep on either side and into each lane's
+//            share of them;
+//   emit     kept indices are staged in shared memory in ascending order, then the group's lanes
+//            write indices and advantages side by side (consecutive lanes, consecutive addresses).
 
-// key at sorted position p of the group (positions are blocked: lane sl holds sl*E .. sl*E+E-1)
-template <int LANES, int E>
-__device__ __forceinline__ uint32_t key_at(const uint32_t (&key)[E], int p, int sub) {
-    uint32_t mine = key[0];
+// reward -> uint32 whose unsigned order is the order of the floats: -0 is folded into +0 by the
+// addition, the sign decides between flipping everything and setting the top bit.  NaNs are dealt
+// with by the caller (they are rare): every NaN gets the key 0xfffffffe, padding 0xffffffff.
+__device__ __forceinline__ uint32_t ordered_key(float r) {
+    const uint32_t u = __float_as_uint(r + 0.0f);
+    return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(uint32_t o) {
+    return __uint_as_float(o ^ (~(uint32_t)((int32_t)o >> 31) | 0x80000000u));
+}
+
+constexpr uint32_t kKeyNaN = 0xfffffffeu;       // above +inf, below the padding
+constexpr uint32_t kKeyPad = 0xffffffffu;
+constexpr uint32_t kKeyNegInf = 0x007fffffu;    // ordered_key(-inf): nothing real sorts below it
+constexpr uint32_t kKeyPosInf = 0xff800000u;    // ordered_key(+inf)
+
+// order-preserving image of a double (NaNs land above or below everything, which is all they need)
+__device__ __forceinline__ unsigned long long ordered_double(double v) {
+    const long long b = __double_as_longlong(v);
+    return (unsigned long long)b ^ ((unsigned long long)(b >> 63) | 0x8000000000000000ull);
+}
+
+// the lowest q set bits of mask (q <= popc(mask)); BITS is the width in use (16 or 32)
+template <int BITS>
+__device__ __forceinline__ uint32_t lowest_set_bits(uint32_t mask, int q) {
+    // L = the largest prefix length whose population is still below q: the q-th set bit is bit L
+    int L = 0;
 #pragma unroll
-    for (int e = 1; e < E; ++e) mine = ((p & (E - 1)) == e) ? key[e] : mine;
-    return __shfl_sync(PODS_FULL_MASK, mine, sub * LANES + ((p / E) & (LANES - 1)));
+    for (int step = BITS / 2; step > 0; step >>= 1) {
+        const int t = L + step;
+        if (__popc(mask & ((1u << t) - 1u)) < q) L = t;
+    }
+    const uint32_t upto = L >= 31 ? 0xffffffffu : ((2u << L) - 1u);
+    return q > 0 ? (mask & upto) : 0u;
 }
 
 template <int LANES, int E>
-__global__ void __launch_bounds__(kSelectThreads, E >= 32 ? 2 : 4)
+__global__ void __launch_bounds__(kSelectThreads, E >= 32 ? 3 : 8)
 pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint32_t flags,
                         int32_t* __restrict__ idx_out, float* __restrict__ adv_out, int32_t* __restrict__ k_out,
                         uint32_t* status) {
     constexpr int NPAD = LANES * E;
     constexpr int GPW = 32 / LANES;                 // groups per warp
+    constexpr int LOGE = E == 4 ? 2 : E == 8 ? 3 : E == 16 ? 4 : 5;
+    constexpr int ROWW = E + 4;                     // words of a lane's row in shared memory
+    constexpr int GROUPW = LANES * ROWW;            // words of a group
+    constexpr uint32_t GROUP_MASK = LANES == 32 ? 0xffffffffu : ((1u << LANES) - 1u);
+    static_assert((1 << LOGE) == E, "E is 4, 8, 16 or 32");
 
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(16) uint32_t smem_words[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / LANES, sl = lane % LANES;
-    double* PL1 = reinterpret_cast<double*>(smem_raw) + (size_t)(warp * GPW + sub) * 4 * (m + 1);   // sum of the j lowest
-    double* PL2 = PL1 + (m + 1);
-    double* SU1 = PL2 + (m + 1);                        // sum of the m-j highest, j = 0..m
-    double* SU2 = SU1 + (m + 1);
-    const bool vec_rows = E % 4 == 0 && (n & 3) == 0 && (reinterpret_cast<uintptr_t>(rewards) & 15) == 0;
+    uint32_t* const ok = smem_words + (size_t)((warp * GPW + sub) * 2) * GROUPW;   // keys in original order
+    uint32_t* const sk = ok + GROUPW;                                               // keys in sorted order
+    int32_t* const stage = reinterpret_cast<int32_t*>(sk);                         // kept indices (sk is dead by then)
+    const uint32_t gmask = GROUP_MASK << (sub * LANES);
+    auto at = [](int p) { return p + ((p >> LOGE) << 2); };                         // word of position p in a group
+    const bool vec_rows = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(rewards) & 15) == 0;
+    const int c = (m + LANES - 1) / LANES;          // sorted positions of each end per lane
+    const int nreal = max(0, min(E, n - sl * E));   // my elements that exist
+    const uint32_t real_mask = nreal >= 32 ? 0xffffffffu : ((1u << nreal) - 1u);
 
     const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
     for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
@@ -348,35 +404,41 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         const bool valid = g < G;
         const float* r_g = rewards + (valid ? g : 0) * (int64_t)n;
 
-        // ---- 1. load and key: lane sl holds original indices sl*E .. sl*E+E-1 (okey keeps that order) ----
-        uint32_t okey[E];
-        bool nonfinite = false;
-        if (vec_rows) {
+        // ---- 1. load and key: lane sl holds original indices sl*E .. sl*E+E-1 -----------------------------
+        uint32_t key[E];
+        {
+            bool nan_seen = false;
+            if (vec_rows) {
 #pragma unroll
-            for (int e = 0; e < E; e += 4) {
-                const int i = sl * E + e;
-                float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                if (i < n && valid) v = *reinterpret_cast<const float4*>(r_g + i);
-                const float f[4] = {v.x, v.y, v.z, v.w};
+                for (int e = 0; e < E; e += 4) {
+                    const int i = sl * E + e;
+                    float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (i < n && valid) v = *reinterpret_cast<const float4*>(r_g + i);
+                    const float f[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    nonfinite |= !(fabsf(f[c]) <= 3.402823466e38f);
-                    okey[e + c < E ? e + c : 0] = i < n ? ordered_bits(f[c]) : 0xffffffffu;
+                    for (int q = 0; q < 4; ++q) {
+                        nan_seen |= f[q] != f[q];
+                        key[e + q] = i < n ? ordered_key(f[q]) : kKeyPad;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const int i = sl * E + e;
+                    const float r = (i < n && valid) ? r_g[i] : 0.0f;
+                    nan_seen |= r != r;
+                    key[e] = i < n ? ordered_key(r) : kKeyPad;
                 }
             }
-        } else {
+            if (__any_sync(PODS_FULL_MASK, nan_seen)) {      // rare: every NaN, whatever its sign, sorts above +inf
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const int i = sl * E + e;
-                const float r = (i < n && valid) ? r_g[i] : 0.0f;
-                nonfinite |= !(fabsf(r) <= 3.402823466e38f);
-                okey[e] = i < n ? ordered_bits(r) : 0xffffffffu;      // padding sorts last (with the NaNs, whose key it shares)
+                for (int e = 0; e < E; ++e)
+                    if (e < nreal && (key[e] > kKeyPosInf || key[e] < kKeyNegInf)) key[e] = kKeyNaN;
             }
         }
-        if (nonfinite && valid) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
-        uint32_t key[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) key[e] = okey[e];
+        for (int e = 0; e < E; e += 4)
+            *reinterpret_cast<uint4*>(ok + sl * ROWW + e) = make_uint4(key[e], key[e + 1], key[e + 2], key[e + 3]);
 
         // ---- 2. bitonic sort of the keys over positions p = sl * E + e ------------------------------
 #pragma unroll
@@ -424,110 +486,131 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
                 }
             }
         }
+#pragma unroll
+        for (int e = 0; e < E; e += 4)
+            *reinterpret_cast<uint4*>(sk + sl * ROWW + e) = make_uint4(key[e], key[e + 1], key[e + 2], key[e + 3]);
+        __syncwarp();
 
-        // ---- 3. centred rewards and fp64 running sums over the sorted order ------------------------
-        const uint32_t first = __shfl_sync(PODS_FULL_MASK, key[0], sub * LANES);
-        const double centre = (double)from_ordered_bits(first);              // the group minimum
-        auto x_of = [&](uint32_t kk, int p) { return p < n ? (double)from_ordered_bits(kk) - centre : 0.0; };
-        int kstar = rule == PODS_RULE_MAXREWARD ? m : 0;                      // m == n: every split is the whole group
-        double k1 = 0.0, k2 = 0.0;                                            // sums of x and x^2 over the kept subset
-        double f1 = 0.0, f2 = 0.0;                                            // ... and over the full group
+        // ---- 3. fp64 running sums of the centred rewards over the two ends of the sorted order ------------
+        const uint32_t k_min = sk[0], k_max = sk[at(n - 1)];
+        const bool nonfinite = k_min <= kKeyNegInf || k_max >= kKeyPosInf;
+        if (nonfinite && valid && sl == 0) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
+        const double centre = (double)key_value(k_min);                      // the group minimum
+        const int j0 = sl * c;                                               // my splits: j0 .. j0 + mine - 1
+        const int mine = max(0, min(c, m - j0));
+        const uint32_t* const lo_keys = sk;                                  // sorted position j      (the j-th lowest)
+        const int hi0 = n - m;                                               // sorted position hi0 + j (the (m-j)-th highest)
+        double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
+#pragma unroll 4
+        for (int i = 0; i < c; ++i) {
+            if (i < mine) {
+                const double xb = (double)key_value(lo_keys[at(j0 + i)]) - centre;
+                const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                sb1 += xb; sb2 += xb * xb;
+                st1 += xt; st2 += xt * xt;
+            }
+        }
+        double below1 = sb1, below2 = sb2;               // inclusive scan over the lanes below (lowest end)
+        double from1 = st1, from2 = st2;                 // inclusive scan over the lanes above (highest end)
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) {
+            const double t1 = __shfl_up_sync(PODS_FULL_MASK, below1, d, LANES);
+            const double t2 = __shfl_up_sync(PODS_FULL_MASK, below2, d, LANES);
+            const double u1 = __shfl_down_sync(PODS_FULL_MASK, from1, d, LANES);
+            const double u2 = __shfl_down_sync(PODS_FULL_MASK, from2, d, LANES);
+            if (sl >= d) { below1 += t1; below2 += t2; }
+            if (sl + d < LANES) { from1 += u1; from2 += u2; }
+        }
+        below1 -= sb1; below2 -= sb2;                    // now: the sum of everything below my first position
+
+        // ---- 4. score my splits: m^2 Var = m * sum x^2 - (sum x)^2; largest score, then largest j -------------
+        // j = number of lowest rewards kept, k = m - j of the highest.  Algorithm 2 starts from k = 0 and
+        // replaces only on a strictly larger variance: among equal scores the largest j wins.
+        const int jforce = rule == PODS_RULE_MAXREWARD ? 0              // all from the top
+                         : (nonfinite || m == n) ? m : -1;              // NaN scores: a scan with '>' stays at k = 0
+        unsigned long long best = 0ull;
+        int bestj = -1;
+        double bq1 = 0.0, bq2 = 0.0;                     // sums over the kept subset of my best split
         {
-            double s1 = 0.0, s2 = 0.0;
-#pragma unroll
+            double a1 = below1, a2 = below2;             // the j lowest, summed upward
+            double b1 = from1, b2 = from2;               // the m-j highest: what is left of the upper end
+            auto consider = [&](int j, double q1, double q2) {
+                // separately rounded products (no fused multiply-add): equal sums give equal scores
+                const unsigned long long s = ordered_double(__dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1)));
+                const bool take = jforce < 0 ? (s >= best) : (j == jforce);
+                if (take) { best = s; bestj = j; bq1 = q1; bq2 = q2; }
+            };
+#pragma unroll 4
+            for (int i = 0; i < c; ++i) {
+                if (i < mine) {
+                    consider(j0 + i, a1 + b1, a2 + b2);
+                    const double xb = (double)key_value(lo_keys[at(j0 + i)]) - centre;
+                    const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                    a1 += xb; a2 += xb * xb;
+                    b1 -= xt; b2 -= xt * xt;
+                }
+            }
+            if (sl == LANES - 1) consider(m, a1, a2);    // the m lowest and none of the highest (k = 0)
+        }
+        int jstar;
+        {
+            const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
+            const uint32_t mh = __reduce_max_sync(gmask, bestj >= 0 ? hi : 0u);
+            bool cand = bestj >= 0 && hi == mh;
+            const uint32_t ml = __reduce_max_sync(gmask, cand ? lo : 0u);
+            cand = cand && lo == ml;
+            const uint32_t mj = __reduce_max_sync(gmask, cand ? (uint32_t)(bestj + 1) : 0u);
+            jstar = mj > 0u ? (int)mj - 1 : m;
+            const uint32_t owners = __ballot_sync(PODS_FULL_MASK, cand && bestj == jstar) & gmask;
+            const int owner = owners ? __ffs(owners) - 1 : lane;
+            bq1 = __shfl_sync(PODS_FULL_MASK, bq1, owner);
+            bq2 = __shfl_sync(PODS_FULL_MASK, bq2, owner);
+        }
+        const int nlo = jstar, nhi = m - jstar;
+        const int kstar = nhi;
+
+        // sums over the whole group, for the "Before" normalisation only
+        double s1 = bq1, s2 = bq2;
+        if (flags & PODS_FLAG_ADV_BEFORE) {
+            double f1 = 0.0, f2 = 0.0;
+#pragma unroll 4
             for (int e = 0; e < E; ++e) {
-                const double x = x_of(key[e], sl * E + e);
-                s1 += x;
-                s2 += x * x;
-            }
-            double i1 = s1, i2 = s2;                         // inclusive scan over the lanes below
-            double j1 = s1, j2 = s2;                         // inclusive scan over the lanes above
-#pragma unroll
-            for (int d = 1; d < LANES; d <<= 1) {
-                const double t1 = __shfl_up_sync(PODS_FULL_MASK, i1, d, LANES);
-                const double t2 = __shfl_up_sync(PODS_FULL_MASK, i2, d, LANES);
-                const double u1 = __shfl_down_sync(PODS_FULL_MASK, j1, d, LANES);
-                const double u2 = __shfl_down_sync(PODS_FULL_MASK, j2, d, LANES);
-                if (sl >= d) { i1 += t1; i2 += t2; }
-                if (sl + d < LANES) { j1 += u1; j2 += u2; }
-            }
-            if (flags & PODS_FLAG_ADV_BEFORE) {
-                f1 = __shfl_sync(PODS_FULL_MASK, i1, sub * LANES + LANES - 1);
-                f2 = __shfl_sync(PODS_FULL_MASK, i2, sub * LANES + LANES - 1);
-            }
-            // Both ends are summed directly (lowest upward, highest downward): no split score is a
-            // difference of running totals, so equal splits score equal and nothing cancels.
-            double a1 = i1 - s1, a2 = i2 - s2;               // sum over positions below this lane's first
-            if (sl * E <= m) {
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int p = sl * E + e;
-                    if (p <= m) { PL1[p] = a1; PL2[p] = a2; }
-                    const double x = x_of(key[e], p);
-                    a1 += x;
-                    a2 += x * x;
-                }
-                if (sl == LANES - 1 && m == NPAD) { PL1[m] = a1; PL2[m] = a2; }   // position m does not exist: the total
-            }
-            double b1 = j1 - s1, b2 = j2 - s2;               // sum over positions above this lane's last
-            if (sl == LANES - 1 && n == NPAD) { SU1[m] = 0.0; SU2[m] = 0.0; }
-            if (sl * E + E - 1 >= n - m) {
-#pragma unroll
-                for (int e = E - 1; e >= 0; --e) {
-                    const int p = sl * E + e;
-                    const double x = x_of(key[e], p);
-                    b1 += x;
-                    b2 += x * x;
-                    if (p >= n - m && p <= n) { SU1[p - (n - m)] = b1; SU2[p - (n - m)] = b2; }
+                if (e < nreal) {
+                    const double x = (double)key_value(sk[sl * ROWW + e]) - centre;
+                    f1 += x; f2 += x * x;
                 }
             }
-            __syncwarp();
-
-            // ---- 4. score the splits: m^2 Var = m * sum x^2 - (sum x)^2 ----------------------------
-            if (rule == PODS_RULE_MAXVAR && m < n) {
-                double best = -INFINITY;
-                int bestk = 0x7fffffff;
-                for (int k = sl; k <= m; k += LANES) {
-                    const double q1 = PL1[m - k] + SU1[m - k];
-                    const double q2 = PL2[m - k] + SU2[m - k];
-                    // separately rounded products (no fused multiply-add): equal sums give equal scores
-                    const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
-                    if (score > best || bestk == 0x7fffffff) { best = score; bestk = k; }
-                }
 #pragma unroll
-                for (int d = LANES >> 1; d > 0; d >>= 1) {
-                    const double ob = __shfl_xor_sync(PODS_FULL_MASK, best, d);
-                    const int ok = __shfl_xor_sync(PODS_FULL_MASK, bestk, d);
-                    if (ok != 0x7fffffff && (bestk == 0x7fffffff || ob > best || (ob == best && ok < bestk))) {
-                        best = ob;
-                        bestk = ok;
-                    }
-                }
-                kstar = __shfl_sync(PODS_FULL_MASK, bestk, sub * LANES);   // one verdict per group, even with NaN scores
+            for (int d = LANES >> 1; d > 0; d >>= 1) {
+                f1 += __shfl_xor_sync(PODS_FULL_MASK, f1, d);
+                f2 += __shfl_xor_sync(PODS_FULL_MASK, f2, d);
             }
-            k1 = PL1[m - kstar] + SU1[m - kstar];
-            k2 = PL2[m - kstar] + SU2[m - kstar];
-            __syncwarp();
+            s1 = f1; s2 = f2;
         }
 
-        // ---- 5. the two thresholds and how many of their ties are kept -------------------------------
-        const int nlo = m - kstar, nhi = kstar;
-        const uint32_t v_lo = key_at<LANES, E>(key, nlo > 0 ? nlo - 1 : 0, sub);
-        const uint32_t v_hi = key_at<LANES, E>(key, nhi > 0 ? n - nhi : 0, sub);
-        // counts over the ORIGINAL order (lane-major = index order), three 10-bit fields in one word:
-        // below v_lo | above v_hi | equal to v_lo | ... ; a group-wide inclusive scan gives totals and,
-        // per lane, how many ties precede it in index order
-        int c_less = 0, c_greater = 0, c_eqlo = 0, c_eqhi = 0;
+        // ---- 5. the two thresholds; my rewards in original order against them ---------------------------
+        // keys of real rewards lie in [1, 0xfffffffe]: 0 and 0xffffffff match nothing when an end is empty
+        const uint32_t v_lo = nlo > 0 ? sk[at(nlo - 1)] : 0u;
+        const uint32_t v_hi = nhi > 0 ? sk[at(n - nhi)] : kKeyPad;
+        __syncwarp();                                    // sk has been read for the last time: it becomes `stage`
+        uint32_t m_lt = 0u, m_el = 0u, m_gt = 0u, m_eh = 0u;
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const bool real = sl * E + e < n;
-            c_less += (real && okey[e] < v_lo) ? 1 : 0;
-            c_greater += (real && okey[e] > v_hi) ? 1 : 0;
-            c_eqlo += (real && okey[e] == v_lo) ? 1 : 0;
-            c_eqhi += (real && okey[e] == v_hi) ? 1 : 0;
+        for (int e = 0; e < E; e += 4) {
+            const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
+            const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                m_lt |= (kk[t] < v_lo ? 1u : 0u) << (e + t);
+                m_el |= (kk[t] == v_lo ? 1u : 0u) << (e + t);
+                m_gt |= (kk[t] > v_hi ? 1u : 0u) << (e + t);
+                m_eh |= (kk[t] == v_hi ? 1u : 0u) << (e + t);
+            }
         }
-        unsigned long long packed = (unsigned long long)c_less | ((unsigned long long)c_greater << 11) |
-                                    ((unsigned long long)c_eqlo << 22) | ((unsigned long long)c_eqhi << 33);
+        m_lt &= real_mask; m_el &= real_mask; m_gt &= real_mask; m_eh &= real_mask;
+        const int c_el = __popc(m_el), c_eh = __popc(m_eh);
+        // four counts of up to 1024 in one word: below v_lo | above v_hi << 11 | equal v_lo << 22 | equal v_hi << 33
+        const unsigned long long packed = (unsigned long long)__popc(m_lt) | ((unsigned long long)__popc(m_gt) << 11) |
+                                          ((unsigned long long)c_el << 22) | ((unsigned long long)c_eh << 33);
         unsigned long long incl = packed;
 #pragma unroll
         for (int d = 1; d < LANES; d <<= 1) {
@@ -538,52 +621,48 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         const unsigned long long before = incl - packed;
         const int need_lo = nlo - (int)(total & 2047);                        // rewards equal to v_lo to keep: the first by index
         const int need_hi = nhi - (int)((total >> 11) & 2047);                // rewards equal to v_hi to keep: the last by index
-        const int first_hi = (int)((total >> 33) & 2047) - need_hi;           // ... i.e. those from this rank on
-        int rank_lo = (int)((before >> 22) & 2047), rank_hi = (int)((before >> 33) & 2047);
-
-        // advantages: a = (x - S/c) / sigma with sigma^2 = (c Q - S^2) / (c d), d = c or c - 1
-        double s1 = k1, s2 = k2;
-        if (flags & PODS_FLAG_ADV_BEFORE) { s1 = f1; s2 = f2; }
-        const double cnt = (flags & PODS_FLAG_ADV_BEFORE) ? (double)n : (double)m;
-        const double den = (flags & PODS_FLAG_STD_SAMPLE) ? cnt - 1.0 : cnt;
-        const double J = __dsub_rn(__dmul_rn(cnt, s2), __dmul_rn(s1, s1));
-        const double inv_sigma_c = (J > 0.0 && den > 0.0) ? sqrt(den / (cnt * J)) : 0.0;   // 1 / (c sigma)
-
-        // ---- 6. which of my rewards are kept; their places in the output (ascending original index) ----
-        uint32_t take_bits = 0u;
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const uint32_t ki = okey[e];
-            const bool in = sl * E + e < n;
-            const bool eq_lo = in && nlo > 0 && ki == v_lo, eq_hi = in && nhi > 0 && ki == v_hi;
-            const bool take = in && ((nlo > 0 && ki < v_lo) || (eq_lo && rank_lo < need_lo) ||
-                                     (nhi > 0 && ki > v_hi) || (eq_hi && rank_hi >= first_hi));
-            take_bits |= take ? (1u << e) : 0u;
-            rank_lo += (in && ki == v_lo) ? 1 : 0;
-            rank_hi += (in && ki == v_hi) ? 1 : 0;
+        const int skip_hi = (int)((total >> 33) & 2047) - need_hi;            // ... i.e. all but the first skip_hi of them
+        const int q_lo = max(0, min(c_el, need_lo - (int)((before >> 22) & 2047)));   // of mine equal to v_lo: keep the first q_lo
+        const int q_hi = max(0, min(c_eh, skip_hi - (int)((before >> 33) & 2047)));   // of mine equal to v_hi: drop the first q_hi
+        uint32_t keep_lo = q_lo == c_el ? m_el : 0u, drop_hi = q_hi == c_eh ? m_eh : 0u;
+        if (__any_sync(PODS_FULL_MASK, (q_lo != 0 && q_lo != c_el) || (q_hi != 0 && q_hi != c_eh))) {
+            keep_lo = lowest_set_bits<E <= 16 ? 16 : 32>(m_el, q_lo);         // a tie run is cut inside some lane
+            drop_hi = lowest_set_bits<E <= 16 ? 16 : 32>(m_eh, q_hi);
         }
-        int my_takes = __popc(take_bits), off = my_takes;
+        const uint32_t take = m_lt | m_gt | keep_lo | (m_eh & ~drop_hi);
+
+        // ---- 6. kept indices in ascending order, then indices and advantages side by side -------------------
+        const int my_takes = __popc(take);
+        int off = my_takes;
 #pragma unroll
         for (int d = 1; d < LANES; d <<= 1) {
             const int t = __shfl_up_sync(PODS_FULL_MASK, off, d, LANES);
             if (sl >= d) off += t;
         }
         off -= my_takes;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if ((take >> e) & 1u) stage[off++] = sl * E + e;
+        }
+        __syncwarp();
+
+        // advantages: a = (x - S/c) / sigma with sigma^2 = (c Q - S^2) / (c d), d = c or c - 1
+        const double cnt = (flags & PODS_FLAG_ADV_BEFORE) ? (double)n : (double)m;
+        const double den = (flags & PODS_FLAG_STD_SAMPLE) ? cnt - 1.0 : cnt;
+        const double J = __dsub_rn(__dmul_rn(cnt, s2), __dmul_rn(s1, s1));
+        const double inv_sigma_c = (J > 0.0 && den > 0.0) ? sqrt(den / (cnt * J)) : 0.0;   // 1 / (c sigma)
         if (valid) {
             int32_t* io = idx_out + g * (int64_t)m;
             float* ao = adv_out + g * (int64_t)m;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                if ((take_bits >> e) & 1u) {
-                    const double xi = (double)from_ordered_bits(okey[e]) - centre;
-                    io[off] = sl * E + e;
-                    ao[off] = (float)((xi * cnt - s1) * inv_sigma_c);
-                    ++off;
-                }
+            for (int j = sl; j < m; j += LANES) {
+                const int i = stage[j] & (NPAD - 1);
+                const double xi = (double)key_value(ok[at(i)]) - centre;
+                io[j] = i;
+                ao[j] = (float)((xi * cnt - s1) * inv_sigma_c);
             }
             if (sl == 0 && k_out != nullptr) k_out[g] = kstar;
         }
-        __syncwarp();
+        __syncwarp();                                    // ok and stage are rewritten by the next group
     }
 }
 
@@ -591,7 +670,8 @@ template <int LANES, int E>
 int launch_select_fast(const float* rewards, int64_t G, int n, int m, int rule, uint32_t flags, int32_t* idx,
                        float* adv, int32_t* k_out, uint32_t* status, cudaStream_t stream) {
     constexpr int GPW = 32 / LANES;
-    const size_t smem = (size_t)4 * (m + 1) * sizeof(double) * kSelectWarps * GPW;
+    // per group: its keys in original and in sorted order, rows of E + 4 words per lane
+    const size_t smem = (size_t)kSelectWarps * GPW * 2 * LANES * (E + 4) * sizeof(uint32_t);
     auto kernel = pods_select_fast_kernel<LANES, E>;
     if (smem > 48 * 1024)
         PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
