@@ -4,7 +4,7 @@
 One step = one pass of the whole path over one batch of synthetic input:
 pods_select -> pods_compact -> grpo_seq_weights -> grpo_loss_chunk per chunk -> grpo_loss_finalize.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--all-configs]
 
 Prints ONE JSON line (rank 0).  `value` is kept tokens per second with every input resident in HBM;
 `e2e` is the same metric through the host-buffer entry point with the copies inside the timed region;
@@ -33,7 +33,28 @@ from paper_2504_13818_b200 import workloads as wl  # noqa: E402
 METRIC = "kept-token GRPO loss+grad tokens/s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-NCU_DRAM_BYTES_PER_ROW = 597643      # ncu capture of grpo_loss_cluster_kernel at V = 151936, see profiles/
+# dram__bytes_read.sum + dram__bytes_write.sum per row of grpo_loss_cluster_kernel<9,9> at V = 151936, from the ncu
+# capture summarised in profiles/grpo_loss_cluster_kernel__c2_profile.md; None once the kernel has changed since
+NCU_DRAM_BYTES_PER_ROW = None
+NCU_CAPTURE_OF = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return {}
+
+
+def loss_kernel_name(V):
+    """The kernel grpo_loss_chunk picks for 16-byte aligned, densely packed rows of V logits."""
+    if V % 8 == 0 and V >= 8192 and V <= 393216:
+        return "grpo_loss_cluster_kernel"
+    if V % 8 == 0 and V <= 4096:
+        return "grpo_loss_tile_kernel"
+    return "grpo_loss_rows_kernel"
 
 
 def parse_args():
@@ -46,6 +67,10 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-select-bench", action="store_true", help="skip the pods_select timings on configs 3 and 4")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long loop of the dominant kernel")
+    ap.add_argument("--no-lm-head", action="store_true", help="skip the fused LM-head log-prob kernel's timing")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="one JSON line with throughput and roofline fractions of all five configs (1 GPU)")
     return ap.parse_args()
 
 

@@ -193,6 +193,28 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
                            void* stream);
 
 /*
+ * grpo_logp_from_hidden - log pi_theta(o_t | p, o_<t), the policy term of L_GRPO (Section 3.1) and L_PODS
+ * (Section 3.2), computed from the last hidden states without ever storing the logits:
+ *   logits[t, :] = hidden[t, :] . W^T  (bf16 inputs, fp32 accumulation on the tensor cores, not rounded to bf16)
+ *   lse[t] = log sum_v exp(logits[t, v])        logp[t] = logits[t, tokens[t]] - lse[t]
+ * This is the forward-only half of fusing the LM-head projection into the objective: it serves the passes that
+ * need no gradient - the frozen sampling policy's old_logp and the reference policy's ref_logp, which
+ * grpo_loss_chunk takes as inputs - and saves them the write and the re-read of [T,V] logits.
+ *
+ *   hidden [dev] bf16 [T, d], row pitch ldh elements      W [dev] bf16 [V, d], row pitch ldw elements
+ *   tokens [dev] int32 [T] (an id outside [0,V) raises PODS_STATUS_TOKEN_RANGE and is read as 0)
+ *   logp   [dev] fp32 [T]                                 lse [dev] fp32 [T] or NULL
+ *   workspace [dev] of grpo_logp_from_hidden_workspace_bytes(T, V, d), 16-byte aligned
+ * Requires d >= 8 and d % 8 == 0, ldh % 8 == 0, ldw % 8 == 0, 16-byte aligned hidden and W (so that every row
+ * starts on a 16-byte boundary); anything else returns PODS_ERR_INVALID_ARG.  Both matrices must live in the
+ * current device's own memory.
+ */
+size_t grpo_logp_from_hidden_workspace_bytes(int64_t T, int32_t V, int32_t d);
+int grpo_logp_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_t ldw, const int32_t* tokens,
+                          int64_t T, int32_t V, int32_t d, float* logp, float* lse, void* workspace,
+                          size_t workspace_bytes, uint32_t* status, void* stream);
+
+/*
  * pods_set_loss_cluster_min_vocab - tuning knob (the paper has no counterpart): grpo_loss_chunk runs rows of
  * V >= min_vocab (V % 8 == 0, 16-byte aligned rows) on the cluster-resident kernel and shorter rows on the
  * row-tile (V <= 4096) or the general row kernel.  The default, 8192, is the measured cross-over on B200; values

@@ -39,6 +39,8 @@ SIGNATURES = {
     "grpo_loss_fwd_bwd": (C.c_int, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i32, _f32, _f32, _i64,
                                     _p, _p, _p, _i64, _p, _sz, _p, _p]),
     "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
+    "grpo_logp_from_hidden_workspace_bytes": (_sz, [_i64, _i32, _i32]),
+    "grpo_logp_from_hidden": (C.c_int, [_p, _i64, _p, _i64, _p, _i64, _i32, _i32, _p, _p, _p, _sz, _p, _p]),
     "pods_selftest_bounded_wait": (C.c_int, [_u32, _p, _p]),
     "pods_set_loss_cluster_min_vocab": (_i32, [_i32]),
     "pods_host_step_create": (C.c_int, [_i64, _i32, _i32, _i64, _i64, _i32, _i64, _p]),
@@ -330,6 +332,42 @@ def grpo_loss_fwd_bwd(logits, tokens, old_logp, ref_logp, adv, mask, eps, beta, 
                                   _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_loss_fwd_bwd")
     return loss, logp, dlogits
+
+
+def grpo_logp_from_hidden_workspace_bytes(T, V, d) -> int:
+    return int(load().grpo_logp_from_hidden_workspace_bytes(T, V, d))
+
+
+def grpo_logp_from_hidden(hidden, W, tokens, logp=None, lse=None, want_lse=False, workspace=None, status=None):
+    """hidden [T,d] bf16, W [V,d] bf16, tokens [T] int32 -> (logp [T] fp32, lse [T] fp32 or None).
+
+    log softmax(hidden W^T)[token] without the logits ever being stored.  Missing outputs and the workspace
+    are allocated here; rows of hidden and W may have a pitch (a column slice of a wider tensor)."""
+    _require(isinstance(hidden, torch.Tensor) and hidden.dim() == 2 and isinstance(W, torch.Tensor) and W.dim() == 2,
+             "hidden must be [T,d] and W [V,d]")
+    T, d = hidden.shape
+    V = W.shape[0]
+    _require(W.shape[1] == d, "W must have d = %d columns, got %d" % (d, W.shape[1]))
+    _numel(tokens, T, "tokens")
+    dev = hidden.device
+    if logp is None:
+        logp = torch.empty(T, dtype=torch.float32, device=dev)
+    if lse is None and want_lse:
+        lse = torch.empty(T, dtype=torch.float32, device=dev)
+    _numel(logp, T, "logp")
+    _numel(lse, T, "lse")
+    need = grpo_logp_from_hidden_workspace_bytes(T, V, d)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    _require(workspace.numel() >= need, "workspace must hold %d bytes, got %d" % (need, workspace.numel()))
+    hp, ldh = _rows(hidden, "hidden")
+    wp, ldw = _rows(W, "W")
+    rc = load().grpo_logp_from_hidden(hp, ldh, wp, ldw, _dev(tokens, torch.int32, "tokens"), T, V, d,
+                                      _dev(logp, torch.float32, "logp"), _dev(lse, torch.float32, "lse", True),
+                                      _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+                                      _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "grpo_logp_from_hidden")
+    return logp, lse
 
 
 class HostStep:

@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise subprocess.CalledProcessError(1, "nvcc -c (%s)" % ", ".join(os.path.basename(f) for f in failed))
     tmp = LIB + ".tmp%d" % os.getpid()
-    subprocess.run([nvcc, "-shared", "-Xcompiler", "-fPIC"] + [obj for obj, _ in jobs] + ["-o", tmp], check=True)
+    subprocess.run([nvcc, "-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a"] + [obj for obj, _ in jobs] + ["-o", tmp], check=True)
     os.replace(tmp, LIB)
     return LIB
 
