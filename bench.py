@@ -268,7 +268,100 @@ def time_select(name, dev, steps, warmup):
     return {"workload": name, "G": w.G, "n": w.n, "m": w.m, "ms": ms, "ms_best": min(times),
             "ms_warm_l2": statistics.median(warm), "groups_per_s": w.G / (ms * 1e-3),
             "GBps": bytes_alg / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": bytes_alg / (ms * 1e-3) / 1e9 / peak,
-            "bound": "alu", "note": "integer ALU pipe at ~65 % of its peak in ncu (profiles/): the sorting network, not HBM"}
+            "bound": "alu", "note": "reads its input once; bound by instruction issue of the per-group sort, scans and "
+                                    "classification (ncu counters in profiles/), not by HBM"}
+
+
+def sustained_loss_kernel(batch, seconds=2.0):
+    """The dominant launch (one full chunk of the fused loss kernel) back to back for `seconds`, with the SM clock
+    sampled meanwhile: the figure under the power cap, beside the burst figure of the step loop."""
+    b, w = batch.b, batch.w
+    rows = batch.chunk
+    lo, hi = 0, rows
+
+    def launch():
+        b.grpo_loss_chunk(batch.logits[lo:hi], batch.tokens[lo:hi], batch.old[lo:hi], batch.ref[lo:hi], batch.adv,
+                          batch.seq_weight, batch.cu, lo, None, w.eps, w.beta, batch.loss_acc, batch.logp[lo:hi],
+                          batch.dlogits[lo:hi], batch.ws, status=batch.status)
+
+    for _ in range(3):
+        launch()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    launch()
+    e1.record()
+    torch.cuda.synchronize()
+    n = max(20, int(seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+    sampler = ClockSampler(batch.dev.index or 0)
+    sampler.start()
+    e0.record()
+    for _ in range(n):
+        launch()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / n
+    bytes_launch = (4 * w.V + 21) * rows
+    achieved = bytes_launch / (ms * 1e-3) / 1e9
+    peak, kind = measured_peak()
+    mhz = clocks.get("sm_mhz")
+    return {"kernel": loss_kernel_name(w.V), "launches": n, "seconds": ms * n * 1e-3, "ms_per_launch": ms,
+            "achieved": achieved, "unit": "GB/s", "peak": peak, "frac": achieved / peak, "peak_kind": "of " + kind,
+            "frac_of_nominal_8TBps": achieved / 8000.0, "sm_mhz_median": mhz,
+            "ms_x_mhz": ms * mhz if mhz else None, "reasons": clocks.get("reasons"),
+            "note": "includes the row-record kernel and the single-CTA reduction of each chunk call"}
+
+
+def time_lm_head(dev, T=16384, V=151936, d=2048, seconds=2.0):
+    """grpo_logp_from_hidden (logits never stored) at the Qwen vocabulary: 2 T V d flop per call against the
+    measured bf16 GEMM rates, timed alone (best of 10) and back to back for `seconds`."""
+    from paper_2504_13818_b200 import binding
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
+    hidden = torch.randn((T, d), generator=gen, device=dev).to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=gen, device=dev) * (3.0 / d ** 0.5)).to(torch.bfloat16)
+    tokens = torch.randint(0, V, (T,), generator=gen, device=dev, dtype=torch.int32)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    ws = torch.empty(binding.grpo_logp_from_hidden_workspace_bytes(T, V, d), dtype=torch.uint8, device=dev)
+    status = binding.new_status(dev)
+
+    def launch():
+        binding.grpo_logp_from_hidden(hidden, W, tokens, logp=logp, workspace=ws, status=status)
+
+    for _ in range(3):
+        launch()
+    torch.cuda.synchronize()
+    alone = []
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        launch()
+        e1.record()
+        torch.cuda.synchronize()
+        alone.append(e0.elapsed_time(e1))
+    n = max(10, int(seconds * 1e3 / min(alone)))
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        launch()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_loop = e0.elapsed_time(e1) / n
+    flop = 2.0 * T * V * d
+    peaks = measured_peaks()
+    burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
+    kind = "of measured" if peaks else "of fallback"
+    return {"kernel": "lm_head_stats_kernel", "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
+            "ms_alone_best": min(alone), "achieved_alone": flop / min(alone) / 1e9, "peak_burst": burst,
+            "frac_alone_of_burst": flop / min(alone) / 1e9 / burst,
+            "ms_loop": ms_loop, "launches": n, "achieved_loop": flop / ms_loop / 1e9, "peak_sustained": sustained,
+            "frac_loop_of_sustained": flop / ms_loop / 1e9 / sustained, "peak_kind": kind,
+            "sm_mhz_median": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
+            "logits_bytes_not_written": 2 * T * V, "device_status_word": binding.read_status(status)}
 
 
 def cpu_baseline(batch, budget_rows=None):
@@ -350,14 +443,19 @@ def run_ours(args):
     bytes_per_token = 4 * w.V + 21
     achieved = bytes_per_token * batch.chunk / (per_launch_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
-    roofline = {"kernel": "grpo_loss_cluster_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+    mhz = clocks.get("sm_mhz") if clocks else None
+    roofline = {"kernel": loss_kernel_name(w.V), "bound": "hbm", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
                 "frac_of_nominal_8TBps": achieved / 8000.0,
-                # dram__bytes_read.sum + dram__bytes_write.sum per launch: 597,643 B per row measured on the 4668-row
-                # capture of this kernel (profiles/), scaled to this launch's rows (traffic is proportional to rows)
-                "traffic": NCU_DRAM_BYTES_PER_ROW * batch.chunk if w.V == 151936 else None,
+                # dram__bytes_read.sum + dram__bytes_write.sum per launch: bytes per row of the ncu capture of this
+                # kernel (profiles/) scaled to this launch's rows (traffic is proportional to rows); None when no
+                # capture of the kernel as it stands exists
+                "traffic": NCU_DRAM_BYTES_PER_ROW * batch.chunk if (NCU_DRAM_BYTES_PER_ROW and w.V == 151936) else None,
+                "traffic_capture": NCU_CAPTURE_OF,
                 "bytes_per_launch": bytes_per_token * batch.chunk, "ms_per_launch": per_launch_ms,
-                "rows_per_launch": batch.chunk}
+                "rows_per_launch": batch.chunk, "sm_mhz_median": mhz,
+                "ms_x_mhz": per_launch_ms * mhz if mhz else None,
+                "timed_region_s": ms_total * 1e-3}
 
     out = {
         "metric": METRIC, "value": whole_job_value(batch.T, args.steps, ms_total, world), "unit": UNIT,
@@ -377,8 +475,12 @@ def run_ours(args):
         out["e2e"] = run_e2e(batch, args)
     else:
         out["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_sustained:
+        out["roofline_sustained"] = sustained_loss_kernel(batch)
     if rank == 0 and world == 1 and not args.no_select_bench:
         out["pods_select"] = [time_select(nm, dev, 20, 3) for nm in ("c3_select_mixed", "c4_select_ties")]
+    if rank == 0 and world == 1 and not args.no_lm_head:
+        out["lm_head"] = time_lm_head(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(batch)
     if rank == 0:
@@ -414,7 +516,22 @@ def run_e2e(batch, args):
 # reference arm: the CPU checker on the host cores
 # --------------------------------------------------------------------------------------------
 
+def reference_rows(w, tokens_rows, rows):
+    """bf16 logits of the first `rows` kept tokens, the ones the GPU arm draws (same generator, same device) when a
+    CUDA device is there; drawn on the host otherwise."""
+    if torch.cuda.is_available() and w.V > 50000:
+        dev = torch.device("cuda:0")
+        tok_d = torch.from_numpy(np.ascontiguousarray(tokens_rows[:2048])).to(dev)
+        lg = wl.make_logits_device(w, tok_d)[:rows]
+        lt = wl.library_logp(lg, tok_d[:rows]).cpu().numpy()
+        return lg.view(torch.uint16).cpu().numpy(), lt, "the GPU arm's first %d rows" % rows
+    logits = wl.make_logits_host(w, tokens_rows[:rows])
+    return logits, wl.host_logp_tilde(logits, tokens_rows[:rows]), "host-drawn rows of the same distribution"
+
+
 def run_reference(args):
+    """The CPU checker, as it stands, on the host cores: each step is selection and compaction in full and the
+    loss + gradient on a bounded sample of the workload's rows."""
     rank, world, _ = dist_env()
     if rank != 0:
         return
@@ -427,8 +544,10 @@ def run_reference(args):
     T = int(cu[-1])
     cores = oracle.num_threads()
     rows = min(T, 48 * cores if w.V > 50000 else 4096)
-    logits = wl.make_logits_host(w, toks[:rows])
-    old, ref = wl.make_old_ref(w, wl.host_logp_tilde(logits, toks[:rows]))
+    logits, lt, drawn = reference_rows(w, toks, rows)
+    noise = np.random.Generator(np.random.PCG64([w.seed, 3]))
+    old = (lt + noise.normal(0.0, w.old_sigma, size=rows)).astype(np.float32)
+    ref = (lt + noise.normal(0.0, w.ref_sigma, size=rows)).astype(np.float32)
     mask = np.ones(T, np.uint8)
     adv32 = sel["adv"].astype(np.float32).reshape(-1)
 
@@ -439,29 +558,104 @@ def run_reference(args):
         o = oracle.grpo_rows(logits, tk[:rows], old, ref, adv32, sw, sor[:rows], mask[:rows], w.eps, w.beta)
         return o
 
-    for _ in range(max(1, min(args.warmup, 1))):
+    for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         step()
     dt = time.perf_counter() - t0
     value = rows * args.steps / dt
-    sample = "each step: select+compact in full (%d groups) and loss+grad on %d of %d rows (V=%d)" % (w.G, rows, T, w.V)
+    sample = ("each step: select+compact in full (%d groups) and loss+grad on %d of %d rows (V=%d; %s)"
+              % (w.G, rows, T, w.V, drawn))
+    chunk = min(w.chunk_rows, T)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "G": w.G, "n": w.n, "m": w.m, "V": w.V, "kept_tokens": T, "rows_per_step": rows},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": {"workload": w.name, "G": w.G, "n": w.n, "m": w.m, "V": w.V, "kept_tokens": T, "chunk_rows": chunk,
+                   "l2": "inputs larger than L2 (logits %.1f GB per step)" % (T * w.V * 2 / 1e9), "replicas": world},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                         "rows_per_step": rows},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+# --------------------------------------------------------------------------------------------
+# all five configs in one record
+# --------------------------------------------------------------------------------------------
+
+def run_all_configs(args):
+    """One JSON line: for each of the five configs the rates of the stages it has (pods_select groups/s; loss +
+    gradient tokens/s), GB/s, both roofline fractions and the CPU checker's rate with its core count."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    import oracle
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    from paper_2504_13818_b200 import binding
+    binding.load()
+    peak, kind = measured_peak()
+    cores = oracle.num_threads()
+    rows_out = []
+    for name in ("c1_tiny", "c2_qwen_vocab", "c3_select_mixed", "c4_select_ties", "c5_large_loss"):
+        w = wl.WORKLOADS[name]
+        entry = {"workload": name, "G": w.G, "n": w.n, "m": w.m, "V": w.V}
+        sel = time_select(name, dev, 30, 5)
+        t0 = time.perf_counter()
+        reps = 3 if w.G * w.n < 1 << 22 else 1
+        for _ in range(reps):
+            oracle.select(_rewards_cache(w), w.m)
+        t_sel = (time.perf_counter() - t0) / reps
+        entry["select"] = {"groups_per_s": sel["groups_per_s"], "us": sel["ms"] * 1e3, "GBps": sel["GBps"],
+                           "frac_of_measured_hbm": sel["frac_of_hbm_peak"], "frac_of_nominal_8TBps": sel["GBps"] / 8000.0,
+                           "oracle_groups_per_s": w.G / t_sel, "oracle_cores": cores}
+        if w.V:
+            batch = Batch(w, dev)
+            steps = 3 if name == "c5_large_loss" else (50 if name == "c1_tiny" else 10)
+            for _ in range(3):
+                batch.step()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                batch.step(record=True)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            loss_ms = sum(a.elapsed_time(b_) for a, b_, _ in batch.loss_events) / steps
+            bytes_step = (4 * w.V + 21) * batch.T
+            base = cpu_baseline(batch, budget_rows=None if w.V > 50000 else min(batch.T, 20000))
+            entry["loss"] = {"kept_tokens": batch.T, "chunks": batch.n_chunks, "kernel": loss_kernel_name(w.V),
+                             "tokens_per_s_step": batch.T / (ms * 1e-3), "ms_per_step": ms,
+                             "tokens_per_s_loss_kernel": batch.T / (loss_ms * 1e-3), "GBps_loss_kernel": bytes_step / (loss_ms * 1e-3) / 1e9,
+                             "frac_of_measured_hbm": bytes_step / (loss_ms * 1e-3) / 1e9 / peak,
+                             "frac_of_nominal_8TBps": bytes_step / (loss_ms * 1e-3) / 1e9 / 8000.0,
+                             "oracle_tokens_per_s": base["value"], "oracle_cores": base["cores"], "oracle_sample": base["sample"],
+                             "loss": float(batch.loss.item()), "device_status_word": binding.read_status(batch.status)}
+            del batch
+            torch.cuda.empty_cache()
+        rows_out.append(entry)
+    print(json.dumps({"all_configs": rows_out, "hbm_peak_GBps": peak, "peak_kind": "of " + kind, "n_gpus": 1,
+                      "data": "synthetic", "timing": "CUDA events; pods_select with L2 flushed between launches; "
+                      "loss inputs larger than L2 except c1_tiny (launch-latency-bound, reported as is)"}))
+
+
+_REWARDS = {}
+
+
+def _rewards_cache(w):
+    if w.name not in _REWARDS:
+        _REWARDS[w.name] = wl.make_rewards(w)
+    return _REWARDS[w.name]
 
 
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.all_configs:
+        run_all_configs(args)
     else:
         run_ours(args)
 
