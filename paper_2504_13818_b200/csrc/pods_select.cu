@@ -372,6 +372,15 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t mask, int q) {
     return q > 0 ? (mask & upto) : 0u;
 }
 
+// all-ones when k < v, from the high word of the 64-bit k - v (neg_v = 0 - v as 64 bits): one multiply-add
+// on the FMA pipe instead of a compare and a select on the integer pipe, which the sort keeps busy.  `one` is a
+// register holding 1 that the compiler cannot see through, so the multiply-add stays one.
+__device__ __forceinline__ uint32_t below_mask(uint32_t k, unsigned long long neg_v, uint32_t one) {
+    unsigned long long d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(k), "r"(one), "l"(neg_v));
+    return (uint32_t)(d >> 32);
+}
+
 template <int LANES, int E>
 __global__ void __launch_bounds__(kSelectThreads, E >= 32 ? 3 : 8)
 pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint32_t flags,
@@ -383,6 +392,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
     constexpr int ROWW = E + 4;                     // words of a lane's row in shared memory
     constexpr int GROUPW = LANES * ROWW;            // words of a group
     constexpr uint32_t GROUP_MASK = LANES == 32 ? 0xffffffffu : ((1u << LANES) - 1u);
+    constexpr int MASK_BITS = E <= 16 ? 16 : 32;
     static_assert((1 << LOGE) == E, "E is 4, 8, 16 or 32");
 
     extern __shared__ __align__(16) uint32_t smem_words[];
@@ -397,6 +407,9 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
     const int c = (m + LANES - 1) / LANES;          // sorted positions of each end per lane
     const int nreal = max(0, min(E, n - sl * E));   // my elements that exist
     const uint32_t real_mask = nreal >= 32 ? 0xffffffffu : ((1u << nreal) - 1u);
+    const float pad_value = __uint_as_float(0x7fffffffu);       // its key is kKeyPad
+    uint32_t one;
+    asm volatile("mov.u32 %0, 1;" : "=r"(one));
 
     const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
     for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
@@ -406,155 +419,180 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
 
         // ---- 1. load and key: lane sl holds original indices sl*E .. sl*E+E-1 -----------------------------
         uint32_t key[E];
-        {
-            bool nan_seen = false;
-            if (vec_rows) {
+        if (vec_rows) {
 #pragma unroll
-                for (int e = 0; e < E; e += 4) {
-                    const int i = sl * E + e;
-                    float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    if (i < n && valid) v = *reinterpret_cast<const float4*>(r_g + i);
-                    const float f[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        nan_seen |= f[q] != f[q];
-                        key[e + q] = i < n ? ordered_key(f[q]) : kKeyPad;
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int i = sl * E + e;
-                    const float r = (i < n && valid) ? r_g[i] : 0.0f;
-                    nan_seen |= r != r;
-                    key[e] = i < n ? ordered_key(r) : kKeyPad;
-                }
+            for (int e = 0; e < E; e += 4) {
+                const int i = sl * E + e;
+                float4 v = make_float4(pad_value, pad_value, pad_value, pad_value);
+                if (i < n) v = valid ? *reinterpret_cast<const float4*>(r_g + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                key[e] = ordered_key(v.x);
+                key[e + 1] = ordered_key(v.y);
+                key[e + 2] = ordered_key(v.z);
+                key[e + 3] = ordered_key(v.w);
             }
-            if (__any_sync(PODS_FULL_MASK, nan_seen)) {      // rare: every NaN, whatever its sign, sorts above +inf
+        } else {
 #pragma unroll
-                for (int e = 0; e < E; ++e)
-                    if (e < nreal && (key[e] > kKeyPosInf || key[e] < kKeyNegInf)) key[e] = kKeyNaN;
+            for (int e = 0; e < E; ++e) {
+                const int i = sl * E + e;
+                key[e] = ordered_key(i < n ? (valid ? r_g[i] : 0.0f) : pad_value);
             }
         }
 #pragma unroll
         for (int e = 0; e < E; e += 4)
             *reinterpret_cast<uint4*>(ok + sl * ROWW + e) = make_uint4(key[e], key[e + 1], key[e + 2], key[e + 3]);
 
-        // ---- 2. bitonic sort of the keys over positions p = sl * E + e ------------------------------
+        // NaNs are not looked for on the way in: after the sort a NaN shows at one end of the order (beyond the
+        // infinities); then, and only then, the group's keys are made canonical and sorted once more.
+        uint32_t k_min, k_max;
+        for (int pass = 0;; ++pass) {
+            // ---- 2. bitonic sort of the keys over positions p = sl * E + e ------------------------------
 #pragma unroll
-        for (int k = 2; k <= NPAD; k <<= 1) {
-            // mirror step: p against p ^ (k - 1)
-            if (k <= E) {
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int f = e ^ (k - 1);
-                    if (e < f) {
-                        const uint32_t a = key[e], b = key[f];
-                        key[e] = min(a, b);
-                        key[f] = max(a, b);
-                    }
-                }
-            } else {
-                const int lane_xor = (k - 1) / E;                      // k / E - 1: all lane bits below k / E
-                const bool lower = (sl & (k / (2 * E))) == 0;
-                uint32_t other[E];
-#pragma unroll
-                for (int e = 0; e < E; ++e) other[e] = __shfl_xor_sync(PODS_FULL_MASK, key[E - 1 - e], lane_xor);
-#pragma unroll
-                for (int e = 0; e < E; ++e) key[e] = lower ? min(key[e], other[e]) : max(key[e], other[e]);
-            }
-            // the remaining steps of the level: p against p ^ j, minimum to the lower position
-#pragma unroll
-            for (int j = k >> 2; j > 0; j >>= 1) {
-                if (j >= E) {
-                    const int lane_xor = j / E;
-                    const bool lower = (sl & lane_xor) == 0;
+            for (int k = 2; k <= NPAD; k <<= 1) {
+                // mirror step: p against p ^ (k - 1)
+                if (k <= E) {
 #pragma unroll
                     for (int e = 0; e < E; ++e) {
-                        const uint32_t other = __shfl_xor_sync(PODS_FULL_MASK, key[e], lane_xor);
-                        key[e] = lower ? min(key[e], other) : max(key[e], other);
+                        const int f = e ^ (k - 1);
+                        if (e < f) {
+                            const uint32_t a = key[e], b = key[f];
+                            key[e] = min(a, b);
+                            key[f] = max(a, b);
+                        }
                     }
                 } else {
+                    const int lane_xor = (k - 1) / E;                      // k / E - 1: all lane bits below k / E
+                    const bool lower = (sl & (k / (2 * E))) == 0;
+                    uint32_t other[E];
 #pragma unroll
-                    for (int e = 0; e < E; ++e) {
-                        if ((e & j) == 0) {
-                            const uint32_t a = key[e], b = key[e | j];
-                            key[e] = min(a, b);
-                            key[e | j] = max(a, b);
+                    for (int e = 0; e < E; ++e) other[e] = __shfl_xor_sync(PODS_FULL_MASK, key[E - 1 - e], lane_xor);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) key[e] = lower ? min(key[e], other[e]) : max(key[e], other[e]);
+                }
+                // the remaining steps of the level: p against p ^ j, minimum to the lower position
+#pragma unroll
+                for (int j = k >> 2; j > 0; j >>= 1) {
+                    if (j >= E) {
+                        const int lane_xor = j / E;
+                        const bool lower = (sl & lane_xor) == 0;
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            const uint32_t other = __shfl_xor_sync(PODS_FULL_MASK, key[e], lane_xor);
+                            key[e] = lower ? min(key[e], other) : max(key[e], other);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if ((e & j) == 0) {
+                                const uint32_t a = key[e], b = key[e | j];
+                                key[e] = min(a, b);
+                                key[e | j] = max(a, b);
+                            }
                         }
                     }
                 }
             }
-        }
 #pragma unroll
-        for (int e = 0; e < E; e += 4)
-            *reinterpret_cast<uint4*>(sk + sl * ROWW + e) = make_uint4(key[e], key[e + 1], key[e + 2], key[e + 3]);
-        __syncwarp();
+            for (int e = 0; e < E; e += 4)
+                *reinterpret_cast<uint4*>(sk + sl * ROWW + e) = make_uint4(key[e], key[e + 1], key[e + 2], key[e + 3]);
+            __syncwarp();
+            k_min = sk[0];
+            k_max = sk[at(n - 1)];
+            const bool stray_nan = k_min < kKeyNegInf || (k_max > kKeyPosInf && k_max != kKeyNaN);
+            if (pass == 1 || !__any_sync(PODS_FULL_MASK, stray_nan)) break;
+            // rare: every NaN, whatever its sign and payload, gets the one key above +inf; back to the sort
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                uint32_t kk = ok[sl * ROWW + e];
+                if (e < nreal && (kk > kKeyPosInf || kk < kKeyNegInf)) kk = kKeyNaN;
+                ok[sl * ROWW + e] = kk;
+                key[e] = kk;
+            }
+            __syncwarp();
+        }
 
         // ---- 3. fp64 running sums of the centred rewards over the two ends of the sorted order ------------
-        const uint32_t k_min = sk[0], k_max = sk[at(n - 1)];
         const bool nonfinite = k_min <= kKeyNegInf || k_max >= kKeyPosInf;
         if (nonfinite && valid && sl == 0) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
         const double centre = (double)key_value(k_min);                      // the group minimum
         const int j0 = sl * c;                                               // my splits: j0 .. j0 + mine - 1
         const int mine = max(0, min(c, m - j0));
-        const uint32_t* const lo_keys = sk;                                  // sorted position j      (the j-th lowest)
-        const int hi0 = n - m;                                               // sorted position hi0 + j (the (m-j)-th highest)
-        double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
-#pragma unroll 4
-        for (int i = 0; i < c; ++i) {
-            if (i < mine) {
-                const double xb = (double)key_value(lo_keys[at(j0 + i)]) - centre;
+        const int hi0 = n - m;                        // sorted position j is the j-th lowest, hi0 + j the (m-j)-th highest
+        // j = number of lowest rewards kept, k = m - j of the highest.  Algorithm 2 starts from k = 0 and replaces
+        // only on a strictly larger variance: among equal scores the largest j wins.
+        const int jforce = rule == PODS_RULE_MAXREWARD ? 0              // all from the top
+                         : (nonfinite || m == n) ? m : -1;              // NaN scores: a scan with '>' stays at k = 0
+        double best = 0.0;
+        int bestj = -1;
+        double bq1 = 0.0, bq2 = 0.0;                  // sums over the kept subset of my best split
+        auto consider = [&](int j, double q1, double q2) {
+            // m^2 Var = m * sum x^2 - (sum x)^2, separately rounded products: equal sums give equal scores
+            const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
+            const bool take = jforce < 0 ? (bestj < 0 || score >= best) : (j == jforce);
+            if (take) { best = score; bestj = j; bq1 = q1; bq2 = q2; }
+        };
+        // one scan over the group: what lies below my lowest-end positions, and the highest end from mine upward
+        auto scan = [&](double sb1, double sb2, double st1, double st2, double& below1, double& below2, double& from1,
+                        double& from2) {
+            below1 = sb1; below2 = sb2; from1 = st1; from2 = st2;
+#pragma unroll
+            for (int d = 1; d < LANES; d <<= 1) {
+                const double t1 = __shfl_up_sync(PODS_FULL_MASK, below1, d, LANES);
+                const double t2 = __shfl_up_sync(PODS_FULL_MASK, below2, d, LANES);
+                const double u1 = __shfl_down_sync(PODS_FULL_MASK, from1, d, LANES);
+                const double u2 = __shfl_down_sync(PODS_FULL_MASK, from2, d, LANES);
+                if (sl >= d) { below1 += t1; below2 += t2; }
+                if (sl + d < LANES) { from1 += u1; from2 += u2; }
+            }
+            below1 -= sb1; below2 -= sb2;
+        };
+        if (c <= 4) {
+            // the usual case (m <= 4 LANES): my values stay in registers between the two sweeps
+            double xb[4], xt[4];
+            double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                xb[i] = 0.0; xt[i] = 0.0;
+                if (i < mine) {
+                    xb[i] = (double)key_value(sk[at(j0 + i)]) - centre;
+                    xt[i] = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                }
+                sb1 += xb[i]; sb2 += xb[i] * xb[i];
+                st1 += xt[i]; st2 += xt[i] * xt[i];
+            }
+            double a1, a2, b1, b2;            // the j lowest, summed upward; the m-j highest: what is left of the upper end
+            scan(sb1, sb2, st1, st2, a1, a2, b1, b2);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (i < mine) consider(j0 + i, a1 + b1, a2 + b2);
+                a1 += xb[i]; a2 += xb[i] * xb[i];
+                b1 -= xt[i]; b2 -= xt[i] * xt[i];
+            }
+            if (sl == LANES - 1) consider(m, a1, a2);    // the m lowest and none of the highest (k = 0)
+        } else {
+            double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
+            for (int i = 0; i < mine; ++i) {
+                const double xb = (double)key_value(sk[at(j0 + i)]) - centre;
                 const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
                 sb1 += xb; sb2 += xb * xb;
                 st1 += xt; st2 += xt * xt;
             }
-        }
-        double below1 = sb1, below2 = sb2;               // inclusive scan over the lanes below (lowest end)
-        double from1 = st1, from2 = st2;                 // inclusive scan over the lanes above (highest end)
-#pragma unroll
-        for (int d = 1; d < LANES; d <<= 1) {
-            const double t1 = __shfl_up_sync(PODS_FULL_MASK, below1, d, LANES);
-            const double t2 = __shfl_up_sync(PODS_FULL_MASK, below2, d, LANES);
-            const double u1 = __shfl_down_sync(PODS_FULL_MASK, from1, d, LANES);
-            const double u2 = __shfl_down_sync(PODS_FULL_MASK, from2, d, LANES);
-            if (sl >= d) { below1 += t1; below2 += t2; }
-            if (sl + d < LANES) { from1 += u1; from2 += u2; }
-        }
-        below1 -= sb1; below2 -= sb2;                    // now: the sum of everything below my first position
-
-        // ---- 4. score my splits: m^2 Var = m * sum x^2 - (sum x)^2; largest score, then largest j -------------
-        // j = number of lowest rewards kept, k = m - j of the highest.  Algorithm 2 starts from k = 0 and
-        // replaces only on a strictly larger variance: among equal scores the largest j wins.
-        const int jforce = rule == PODS_RULE_MAXREWARD ? 0              // all from the top
-                         : (nonfinite || m == n) ? m : -1;              // NaN scores: a scan with '>' stays at k = 0
-        unsigned long long best = 0ull;
-        int bestj = -1;
-        double bq1 = 0.0, bq2 = 0.0;                     // sums over the kept subset of my best split
-        {
-            double a1 = below1, a2 = below2;             // the j lowest, summed upward
-            double b1 = from1, b2 = from2;               // the m-j highest: what is left of the upper end
-            auto consider = [&](int j, double q1, double q2) {
-                // separately rounded products (no fused multiply-add): equal sums give equal scores
-                const unsigned long long s = ordered_double(__dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1)));
-                const bool take = jforce < 0 ? (s >= best) : (j == jforce);
-                if (take) { best = s; bestj = j; bq1 = q1; bq2 = q2; }
-            };
-#pragma unroll 4
-            for (int i = 0; i < c; ++i) {
-                if (i < mine) {
-                    consider(j0 + i, a1 + b1, a2 + b2);
-                    const double xb = (double)key_value(lo_keys[at(j0 + i)]) - centre;
-                    const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
-                    a1 += xb; a2 += xb * xb;
-                    b1 -= xt; b2 -= xt * xt;
-                }
+            double a1, a2, b1, b2;
+            scan(sb1, sb2, st1, st2, a1, a2, b1, b2);
+            for (int i = 0; i < mine; ++i) {
+                consider(j0 + i, a1 + b1, a2 + b2);
+                const double xb = (double)key_value(sk[at(j0 + i)]) - centre;
+                const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                a1 += xb; a2 += xb * xb;
+                b1 -= xt; b2 -= xt * xt;
             }
-            if (sl == LANES - 1) consider(m, a1, a2);    // the m lowest and none of the highest (k = 0)
+            if (sl == LANES - 1) consider(m, a1, a2);
         }
+
+        // ---- 4. arg-max over the group: largest score, then largest j --------------------------------------
         int jstar;
         {
-            const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
+            const unsigned long long ob = ordered_double(best);
+            const uint32_t hi = (uint32_t)(ob >> 32), lo = (uint32_t)ob;
             const uint32_t mh = __reduce_max_sync(gmask, bestj >= 0 ? hi : 0u);
             bool cand = bestj >= 0 && hi == mh;
             const uint32_t ml = __reduce_max_sync(gmask, cand ? lo : 0u);
@@ -592,44 +630,65 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         // keys of real rewards lie in [1, 0xfffffffe]: 0 and 0xffffffff match nothing when an end is empty
         const uint32_t v_lo = nlo > 0 ? sk[at(nlo - 1)] : 0u;
         const uint32_t v_hi = nhi > 0 ? sk[at(n - nhi)] : kKeyPad;
+        // a run of equal rewards is cut when the sorted neighbour just outside a kept end has the end's value
+        const bool cut = (nlo > 0 && nlo < n && sk[at(nlo)] == v_lo) || (nhi > 0 && nhi < n && sk[at(n - nhi - 1)] == v_hi);
         __syncwarp();                                    // sk has been read for the last time: it becomes `stage`
-        uint32_t m_lt = 0u, m_el = 0u, m_gt = 0u, m_eh = 0u;
+        uint32_t take = 0u;
+        if (!__any_sync(PODS_FULL_MASK, cut)) {
+            // no run is cut anywhere in the warp: everything up to v_lo and everything from v_hi on is kept
 #pragma unroll
-        for (int e = 0; e < E; e += 4) {
-            const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
-            const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
+            for (int e = 0; e < E; e += 4) {
+                const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
+                const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                m_lt |= (kk[t] < v_lo ? 1u : 0u) << (e + t);
-                m_el |= (kk[t] == v_lo ? 1u : 0u) << (e + t);
-                m_gt |= (kk[t] > v_hi ? 1u : 0u) << (e + t);
-                m_eh |= (kk[t] == v_hi ? 1u : 0u) << (e + t);
+                for (int t = 0; t < 4; ++t) take |= ((kk[t] <= v_lo || kk[t] >= v_hi) ? 1u : 0u) << (e + t);
             }
-        }
-        m_lt &= real_mask; m_el &= real_mask; m_gt &= real_mask; m_eh &= real_mask;
-        const int c_el = __popc(m_el), c_eh = __popc(m_eh);
-        // four counts of up to 1024 in one word: below v_lo | above v_hi << 11 | equal v_lo << 22 | equal v_hi << 33
-        const unsigned long long packed = (unsigned long long)__popc(m_lt) | ((unsigned long long)__popc(m_gt) << 11) |
-                                          ((unsigned long long)c_el << 22) | ((unsigned long long)c_eh << 33);
-        unsigned long long incl = packed;
+            take &= real_mask;
+        } else {
+            // four masks over my rewards: below v_lo, up to v_lo, below v_hi, up to v_hi
+            const unsigned long long neg_lo = 0ull - (unsigned long long)v_lo, neg_hi = 0ull - (unsigned long long)v_hi;
+            uint32_t m_lt = 0u, m_le = 0u, m_lth = 0u, m_leh = 0u;
 #pragma unroll
-        for (int d = 1; d < LANES; d <<= 1) {
-            const unsigned long long t = __shfl_up_sync(PODS_FULL_MASK, incl, d, LANES);
-            if (sl >= d) incl += t;
+            for (int e = 0; e < E; e += 4) {
+                const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
+                const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t bit = 1u << (e + t);
+                    m_lt |= below_mask(kk[t], neg_lo, one) & bit;
+                    m_le |= below_mask(kk[t], neg_lo - 1ull, one) & bit;
+                    m_lth |= below_mask(kk[t], neg_hi, one) & bit;
+                    m_leh |= below_mask(kk[t], neg_hi - 1ull, one) & bit;
+                }
+            }
+            m_lt &= real_mask;
+            const uint32_t m_el = m_le & ~m_lt & real_mask;              // equal to v_lo
+            const uint32_t m_gt = ~m_leh & real_mask;                    // above v_hi
+            const uint32_t m_eh = m_leh & ~m_lth & real_mask;            // equal to v_hi
+            const int c_el = __popc(m_el), c_eh = __popc(m_eh);
+            // four counts of up to 1024 in one word: below v_lo | above v_hi << 11 | equal v_lo << 22 | equal v_hi << 33
+            const unsigned long long packed = (unsigned long long)__popc(m_lt) | ((unsigned long long)__popc(m_gt) << 11) |
+                                              ((unsigned long long)c_el << 22) | ((unsigned long long)c_eh << 33);
+            unsigned long long incl = packed;
+#pragma unroll
+            for (int d = 1; d < LANES; d <<= 1) {
+                const unsigned long long t = __shfl_up_sync(PODS_FULL_MASK, incl, d, LANES);
+                if (sl >= d) incl += t;
+            }
+            const unsigned long long total = __shfl_sync(PODS_FULL_MASK, incl, sub * LANES + LANES - 1);
+            const unsigned long long before = incl - packed;
+            const int need_lo = nlo - (int)(total & 2047);                        // rewards equal to v_lo to keep: the first by index
+            const int need_hi = nhi - (int)((total >> 11) & 2047);                // rewards equal to v_hi to keep: the last by index
+            const int skip_hi = (int)((total >> 33) & 2047) - need_hi;            // ... i.e. all but the first skip_hi of them
+            const int q_lo = max(0, min(c_el, need_lo - (int)((before >> 22) & 2047)));   // of mine equal to v_lo: keep the first q_lo
+            const int q_hi = max(0, min(c_eh, skip_hi - (int)((before >> 33) & 2047)));   // of mine equal to v_hi: drop the first q_hi
+            uint32_t keep_lo = q_lo == c_el ? m_el : 0u, drop_hi = q_hi == c_eh ? m_eh : 0u;
+            if (__any_sync(PODS_FULL_MASK, (q_lo != 0 && q_lo != c_el) || (q_hi != 0 && q_hi != c_eh))) {
+                keep_lo = lowest_set_bits<MASK_BITS>(m_el, q_lo);                 // the cut falls inside some lane
+                drop_hi = lowest_set_bits<MASK_BITS>(m_eh, q_hi);
+            }
+            take = m_lt | m_gt | keep_lo | (m_eh & ~drop_hi);
         }
-        const unsigned long long total = __shfl_sync(PODS_FULL_MASK, incl, sub * LANES + LANES - 1);
-        const unsigned long long before = incl - packed;
-        const int need_lo = nlo - (int)(total & 2047);                        // rewards equal to v_lo to keep: the first by index
-        const int need_hi = nhi - (int)((total >> 11) & 2047);                // rewards equal to v_hi to keep: the last by index
-        const int skip_hi = (int)((total >> 33) & 2047) - need_hi;            // ... i.e. all but the first skip_hi of them
-        const int q_lo = max(0, min(c_el, need_lo - (int)((before >> 22) & 2047)));   // of mine equal to v_lo: keep the first q_lo
-        const int q_hi = max(0, min(c_eh, skip_hi - (int)((before >> 33) & 2047)));   // of mine equal to v_hi: drop the first q_hi
-        uint32_t keep_lo = q_lo == c_el ? m_el : 0u, drop_hi = q_hi == c_eh ? m_eh : 0u;
-        if (__any_sync(PODS_FULL_MASK, (q_lo != 0 && q_lo != c_el) || (q_hi != 0 && q_hi != c_eh))) {
-            keep_lo = lowest_set_bits<E <= 16 ? 16 : 32>(m_el, q_lo);         // a tie run is cut inside some lane
-            drop_hi = lowest_set_bits<E <= 16 ? 16 : 32>(m_eh, q_hi);
-        }
-        const uint32_t take = m_lt | m_gt | keep_lo | (m_eh & ~drop_hi);
 
         // ---- 6. kept indices in ascending order, then indices and advantages side by side -------------------
         const int my_takes = __popc(take);
