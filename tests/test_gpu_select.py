@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2504_13818_b200 import binding, workloads as wl
-from parity import assert_adv_close, shrink
+from parity import assert_adv_close, record, shrink
 
 pytestmark = pytest.mark.gpu
 
@@ -38,6 +38,10 @@ def _reward_kinds(rng, G, n):
     yield "mixed", (rng.integers(0, 2, (G, n)) + 0.1 * rng.integers(0, 2, (G, n))
                     + rng.normal(0, 0.05, (G, n))).astype(np.float32)
     yield "negatives", rng.choice([-2.0, -0.25, 0.0, 0.25, 3.0], (G, n)).astype(np.float32)
+    # values that are not dyadic: sums of their squares are not exact in fp64, yet splits that keep the same
+    # multiset of rewards must still tie (an accuracy reward of 1 plus a format credit of 0.1, as in Appendix A.1)
+    yield "decimal", rng.choice([0.1, 0.3, 0.7], (G, n)).astype(np.float32)
+    yield "accuracy+format", (rng.integers(0, 2, (G, n)) + 0.1 * rng.integers(0, 2, (G, n))).astype(np.float32)
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 7, 8, 9, 16, 17, 31, 32, 33, 48, 64, 100, 128, 200, 256, 257, 512, 1000, 1024])
@@ -53,7 +57,12 @@ def test_every_kernel_shape_and_ragged_n(n):
 def test_workload_rewards_at_full_size():
     for name in ("c1_tiny", "c2_qwen_vocab", "c3_select_mixed", "c4_select_ties", "c5_large_loss"):
         w = wl.WORKLOADS[name]
-        _compare(wl.make_rewards(w), w.m)
+        r = wl.make_rewards(w)
+        idx, adv, k = _compare(r, w.m)                   # indices and k bit-exact, advantages within tolerance
+        want = oracle.select(r, w.m)["adv"]
+        nz = want != 0
+        rel = float((np.abs(adv.astype(np.float64) - want)[nz] / np.abs(want[nz])).max()) if nz.any() else 0.0
+        record("%s rewards at full size (G=%d, n=%d, m=%d)" % (name, w.G, w.n, w.m), idx_exact=1, adv_rel=rel)
 
 
 def test_degenerate_and_special_values():
