@@ -59,6 +59,7 @@ typedef enum {
 
 #define PODS_FLAG_ADV_BEFORE 0x1u  /* advantages from full-group statistics (Appendix A.3 "Before") */
 #define PODS_FLAG_STD_SAMPLE 0x2u  /* divide by (count-1) instead of count in the standard deviation  */
+#define PODS_FLAG_EXACT_TIES 0x4u  /* max-variance rule: settle near-equal split scores in ~106-bit arithmetic (see pods_select) */
 
 #define PODS_MAX_N 1024            /* largest supported group size n */
 
@@ -76,6 +77,12 @@ int pods_read_status(const uint32_t* status /*dev*/, uint32_t* host_value /*host
  * rewards (ties by index, -0 == +0), and over k = 0..m take the k highest and m-k lowest whose
  * variance is largest, the smallest such k on ties (Algorithm 2 replaces only on a strictly
  * larger variance).  Split scores are evaluated in fp64 on rewards centred on the group minimum.
+ * Ties: splits that keep the same multiset of rewards, and the mirror pair of a two-valued kept subset
+ * (j of a and m-j of b against m-j of a and j of b), tie for any reward values and are recognised from the
+ * sorted rewards themselves; these are the only ties that do not depend on the values.  Every other tie is
+ * decided by the fp64 scores, which is exact whenever the sums are (rewards on a coarse dyadic grid such as
+ * {0, 0.5, 1}) but not for coincidences among rewards like 0.1, 0.2, 0.4; PODS_FLAG_EXACT_TIES re-evaluates
+ * such near-ties in double-double arithmetic (about 10 % slower).
  * PODS_RULE_RANDOM keeps the m rollouts with the smallest 32-bit Philox4x32-10 words (counter
  * (i, 0, g lo, g hi), key = seed, first output word; ties by index).  PODS_RULE_PERCENTILE keeps
  * sorted positions floor((j+0.5) n/m), j = 0..m-1.

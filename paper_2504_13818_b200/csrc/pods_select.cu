@@ -372,6 +372,119 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t mask, int q) {
     return q > 0 ? (mask & upto) : 0u;
 }
 
+// ---- exact arg-max over the splits, for groups whose fp64 scores cannot decide --------------------------------
+// A score m sum x^2 - (sum x)^2 of fp32 rewards needs up to ~75 bits; fp64 rounds it, and splits that tie exactly
+// in real arithmetic (two kept values a < b: j of a and m-j of b score j (m-j) (b-a)^2, the same for j and m-j)
+// come out a few ulps apart unless every sum happens to be exact (dyadic rewards).  When the fp64 scores leave a
+// rival within 2^-40 of the best outside the best's own run of identical multisets, the group's scores are
+// evaluated again here in double-double arithmetic (two fp64 words, ~106 bits: error-free products by fused
+// multiply-add, sums by the branch-free two-sum), and scores closer than 2^-90 relative count as equal: exact for
+// rewards whose magnitudes lie within ~2^11 of each other beyond their 24 bits, far below any rounding otherwise.
+struct dd { double hi, lo; };
+__device__ __forceinline__ dd two_sum(double a, double b) {
+    const double s = __dadd_rn(a, b), bb = __dsub_rn(s, a);
+    return {s, __dadd_rn(__dsub_rn(a, __dsub_rn(s, bb)), __dsub_rn(b, bb))};
+}
+__device__ __forceinline__ dd quick_two_sum(double a, double b) {          // |a| >= |b|
+    const double s = __dadd_rn(a, b);
+    return {s, __dsub_rn(b, __dsub_rn(s, a))};
+}
+__device__ __forceinline__ dd dd_add(dd x, dd y) {
+    dd s = two_sum(x.hi, y.hi);
+    const dd t = two_sum(x.lo, y.lo);
+    s = quick_two_sum(s.hi, __dadd_rn(s.lo, t.hi));
+    return quick_two_sum(s.hi, __dadd_rn(s.lo, t.lo));
+}
+__device__ __forceinline__ dd dd_sub(dd x, dd y) { return dd_add(x, {-y.hi, -y.lo}); }
+__device__ __forceinline__ dd dd_add_d(dd x, double d) { return dd_add(x, {d, 0.0}); }
+__device__ __forceinline__ dd dd_square_d(double a) {
+    const double p = __dmul_rn(a, a);
+    return {p, __fma_rn(a, a, -p)};
+}
+__device__ __forceinline__ dd dd_mul(dd x, dd y) {
+    const double p = __dmul_rn(x.hi, y.hi);
+    double e = __fma_rn(x.hi, y.hi, -p);
+    e = __fma_rn(x.hi, y.lo, e);
+    e = __fma_rn(x.lo, y.hi, e);
+    return quick_two_sum(p, e);
+}
+__device__ __forceinline__ dd dd_mul_d(dd x, double d) {
+    const double p = __dmul_rn(x.hi, d);
+    return quick_two_sum(p, __fma_rn(x.lo, d, __fma_rn(x.hi, d, -p)));
+}
+__device__ __forceinline__ dd dd_shfl(dd v, int src) {
+    return {__shfl_sync(PODS_FULL_MASK, v.hi, src), __shfl_sync(PODS_FULL_MASK, v.lo, src)};
+}
+// a >= b up to 2^-90 of the larger: the scores are non-negative up to rounding
+__device__ __forceinline__ bool dd_not_below(dd a, dd b) {
+    const dd d = dd_sub(a, b);
+    const double diff = __dadd_rn(d.hi, d.lo);
+    return diff >= -ldexp(fmax(fabs(a.hi), fabs(b.hi)), -90);
+}
+
+// Every lane of the warp calls this together.  Returns the exact jstar of the lane's group (the largest j among
+// the splits of maximal score) and the sums of x and x^2 over that split's kept subset.
+template <int LANES, int LOGE>
+__device__ __noinline__ int exact_best_split(const uint32_t* sk, int n, int m, int c, int sub, int sl, uint32_t gmask,
+                                             double centre, double* q1_out, double* q2_out) {
+    auto at = [](int p) { return p + ((p >> LOGE) << 2); };
+    const int j0 = sl * c, mine = max(0, min(c, m - j0)), hi0 = n - m;
+    auto x_at = [&](int p) {
+        const uint32_t o = sk[at(p)];
+        return (double)__uint_as_float(o ^ (~(uint32_t)((int32_t)o >> 31) | 0x80000000u)) - centre;
+    };
+    dd sb1 = {0.0, 0.0}, sb2 = sb1, st1 = sb1, st2 = sb1;
+    for (int i = 0; i < mine; ++i) {
+        const double xb = x_at(j0 + i), xt = x_at(hi0 + j0 + i);
+        sb1 = dd_add_d(sb1, xb); sb2 = dd_add(sb2, dd_square_d(xb));
+        st1 = dd_add_d(st1, xt); st2 = dd_add(st2, dd_square_d(xt));
+    }
+    dd a1 = sb1, a2 = sb2, b1 = st1, b2 = st2;       // inclusive scans: the lanes below / from mine upward
+#pragma unroll
+    for (int d = 1; d < LANES; d <<= 1) {
+        const int up = (sub * LANES) + max(sl - d, 0), down = (sub * LANES) + min(sl + d, LANES - 1);
+        const dd t1 = dd_shfl(a1, up), t2 = dd_shfl(a2, up), u1 = dd_shfl(b1, down), u2 = dd_shfl(b2, down);
+        if (sl >= d) { a1 = dd_add(a1, t1); a2 = dd_add(a2, t2); }
+        if (sl + d < LANES) { b1 = dd_add(b1, u1); b2 = dd_add(b2, u2); }
+    }
+    a1 = dd_sub(a1, sb1); a2 = dd_sub(a2, sb2);
+    dd best = {0.0, 0.0}, bq1 = best, bq2 = best;
+    int bestj = -1;
+    auto consider = [&](int j, dd q1, dd q2) {
+        const dd score = dd_sub(dd_mul_d(q2, (double)m), dd_mul(q1, q1));
+        if (bestj < 0 || dd_not_below(score, best)) {
+            // keep the larger of the two as the reference, so that a chain of near-equal scores cannot drift
+            if (bestj < 0 || !dd_not_below(best, score)) best = score;
+            bestj = j; bq1 = q1; bq2 = q2;
+        }
+    };
+    for (int i = 0; i < mine; ++i) {
+        consider(j0 + i, dd_add(a1, b1), dd_add(a2, b2));
+        const double xb = x_at(j0 + i), xt = x_at(hi0 + j0 + i);
+        a1 = dd_add_d(a1, xb); a2 = dd_add(a2, dd_square_d(xb));
+        b1 = dd_add_d(b1, -xt); b2 = dd_sub(b2, dd_square_d(xt));
+    }
+    if (sl == LANES - 1) consider(m, a1, a2);
+    // the group's largest score (by its high word; words below that are inside the tolerance), then every lane
+    // whose best is not below it competes with its j
+    const unsigned long long ob = ordered_double(best.hi);
+    const uint32_t hi = (uint32_t)(ob >> 32), lo = (uint32_t)ob;
+    const uint32_t mh = __reduce_max_sync(gmask, bestj >= 0 ? hi : 0u);
+    bool cand = bestj >= 0 && hi == mh;
+    const uint32_t ml = __reduce_max_sync(gmask, cand ? lo : 0u);
+    cand = cand && lo == ml;
+    const uint32_t tops = __ballot_sync(PODS_FULL_MASK, cand) & gmask;
+    const dd top = dd_shfl(best, tops ? __ffs(tops) - 1 : (sub * LANES));
+    const bool in = bestj >= 0 && dd_not_below(best, top);
+    const uint32_t mj = __reduce_max_sync(gmask, in ? (uint32_t)(bestj + 1) : 0u);
+    const int jstar = mj > 0u ? (int)mj - 1 : m;
+    const uint32_t owners = __ballot_sync(PODS_FULL_MASK, in && bestj == jstar) & gmask;
+    const int owner = owners ? __ffs(owners) - 1 : (sub * LANES);
+    *q1_out = __shfl_sync(PODS_FULL_MASK, bq1.hi, owner);
+    *q2_out = __shfl_sync(PODS_FULL_MASK, bq2.hi, owner);
+    return jstar;
+}
+
 // all-ones when k < v, from the high word of the 64-bit k - v (neg_v = 0 - v as 64 bits): one multiply-add
 // on the FMA pipe instead of a compare and a select on the integer pipe, which the sort keeps busy.  `one` is a
 // register holding 1 that the compiler cannot see through, so the multiply-add stays one.
@@ -381,7 +494,50 @@ __device__ __forceinline__ uint32_t below_mask(uint32_t k, unsigned long long ne
     return (uint32_t)(d >> 32);
 }
 
-template <int LANES, int E>
+// A lane's standing among its own splits: the best score so far with its j and the sums over its kept subset, and
+// the best score among its splits that keep another multiset than that best (`run` numbers the runs of identical
+// multisets among the lane's splits): a rival the fp64 scores may fail to separate from the winner.
+struct SplitBest {
+    double best, q1, q2, runner_up;
+    int j, run;
+};
+
+// m^2 Var = m * sum x^2 - (sum x)^2 of the split "j lowest + (m - j) highest" whose kept subset sums to q1, q2;
+// separately rounded products, so that equal sums give equal scores.  The later of two equal scores leads.
+template <bool EXACT>
+__device__ __forceinline__ void consider_split(SplitBest& s, int jforce, int m, int j, int run, double q1, double q2) {
+    const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
+    const bool take = jforce < 0 ? (s.j < 0 || score >= s.best) : (j == jforce);
+    if (EXACT) {
+        const bool other_run = s.j >= 0 && run != s.run;
+        const double loser = take ? s.best : score;             // the one of the two that does not lead
+        s.runner_up = other_run ? fmax(s.runner_up, loser) : s.runner_up;
+    }
+    s.best = take ? score : s.best;
+    s.q1 = take ? q1 : s.q1;
+    s.q2 = take ? q2 : s.q2;
+    s.j = take ? j : s.j;
+    s.run = take ? run : s.run;
+}
+
+// One scan over the group's LANES lanes: (b1, b2) -> the sums of the lanes below; (t1, t2) -> the sums from this
+// lane upward.
+template <int LANES>
+__device__ __forceinline__ void scan_both_ends(int sl, double& b1, double& b2, double& t1, double& t2) {
+    const double own1 = b1, own2 = b2;
+#pragma unroll
+    for (int d = 1; d < LANES; d <<= 1) {
+        const double p1 = __shfl_up_sync(PODS_FULL_MASK, b1, d, LANES);
+        const double p2 = __shfl_up_sync(PODS_FULL_MASK, b2, d, LANES);
+        const double u1 = __shfl_down_sync(PODS_FULL_MASK, t1, d, LANES);
+        const double u2 = __shfl_down_sync(PODS_FULL_MASK, t2, d, LANES);
+        if (sl >= d) { b1 += p1; b2 += p2; }
+        if (sl + d < LANES) { t1 += u1; t2 += u2; }
+    }
+    b1 -= own1; b2 -= own2;
+}
+
+template <int LANES, int E, bool EXACT>
 __global__ void __launch_bounds__(kSelectThreads, E >= 32 ? 3 : 8)
 pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, int rule, uint32_t flags,
                         int32_t* __restrict__ idx_out, float* __restrict__ adv_out, int32_t* __restrict__ k_out,
@@ -521,72 +677,56 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         // only on a strictly larger variance: among equal scores the largest j wins.
         const int jforce = rule == PODS_RULE_MAXREWARD ? 0              // all from the top
                          : (nonfinite || m == n) ? m : -1;              // NaN scores: a scan with '>' stays at k = 0
-        double best = 0.0;
-        int bestj = -1;
-        double bq1 = 0.0, bq2 = 0.0;                  // sums over the kept subset of my best split
-        auto consider = [&](int j, double q1, double q2) {
-            // m^2 Var = m * sum x^2 - (sum x)^2, separately rounded products: equal sums give equal scores
-            const double score = __dsub_rn(__dmul_rn((double)m, q2), __dmul_rn(q1, q1));
-            const bool take = jforce < 0 ? (bestj < 0 || score >= best) : (j == jforce);
-            if (take) { best = score; bestj = j; bq1 = q1; bq2 = q2; }
-        };
-        // one scan over the group: what lies below my lowest-end positions, and the highest end from mine upward
-        auto scan = [&](double sb1, double sb2, double st1, double st2, double& below1, double& below2, double& from1,
-                        double& from2) {
-            below1 = sb1; below2 = sb2; from1 = st1; from2 = st2;
-#pragma unroll
-            for (int d = 1; d < LANES; d <<= 1) {
-                const double t1 = __shfl_up_sync(PODS_FULL_MASK, below1, d, LANES);
-                const double t2 = __shfl_up_sync(PODS_FULL_MASK, below2, d, LANES);
-                const double u1 = __shfl_down_sync(PODS_FULL_MASK, from1, d, LANES);
-                const double u2 = __shfl_down_sync(PODS_FULL_MASK, from2, d, LANES);
-                if (sl >= d) { below1 += t1; below2 += t2; }
-                if (sl + d < LANES) { from1 += u1; from2 += u2; }
-            }
-            below1 -= sb1; below2 -= sb2;
-        };
+        SplitBest sb = {0.0, 0.0, 0.0, -INFINITY, -1, -1};
+        uint32_t differs = 0u;                        // bit i: splits j0+i and j0+i+1 keep different multisets
         if (c <= 4) {
             // the usual case (m <= 4 LANES): my values stay in registers between the two sweeps
             double xb[4], xt[4];
-            double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
+            double a1 = 0.0, a2 = 0.0, b1 = 0.0, b2 = 0.0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 xb[i] = 0.0; xt[i] = 0.0;
                 if (i < mine) {
-                    xb[i] = (double)key_value(sk[at(j0 + i)]) - centre;
-                    xt[i] = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                    const uint32_t kb = sk[at(j0 + i)], kt = sk[at(hi0 + j0 + i)];
+                    differs |= (kb != kt ? 1u : 0u) << i;
+                    xb[i] = (double)key_value(kb) - centre;
+                    xt[i] = (double)key_value(kt) - centre;
                 }
-                sb1 += xb[i]; sb2 += xb[i] * xb[i];
-                st1 += xt[i]; st2 += xt[i] * xt[i];
+                a1 += xb[i]; a2 += xb[i] * xb[i];
+                b1 += xt[i]; b2 += xt[i] * xt[i];
             }
-            double a1, a2, b1, b2;            // the j lowest, summed upward; the m-j highest: what is left of the upper end
-            scan(sb1, sb2, st1, st2, a1, a2, b1, b2);
+            // a: the j lowest, summed upward; b: the m-j highest, i.e. what is left of the upper end
+            scan_both_ends<LANES>(sl, a1, a2, b1, b2);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                if (i < mine) consider(j0 + i, a1 + b1, a2 + b2);
+                if (i < mine) consider_split<EXACT>(sb, jforce, m, j0 + i, (EXACT ? __popc(differs & ((1u << i) - 1u)) : 0), a1 + b1, a2 + b2);
                 a1 += xb[i]; a2 += xb[i] * xb[i];
                 b1 -= xt[i]; b2 -= xt[i] * xt[i];
             }
-            if (sl == LANES - 1) consider(m, a1, a2);    // the m lowest and none of the highest (k = 0)
+            if (sl == LANES - 1) consider_split<EXACT>(sb, jforce, m, m, (EXACT ? __popc(differs) : 0), a1, a2);   // the m lowest, none of the highest
         } else {
-            double sb1 = 0.0, sb2 = 0.0, st1 = 0.0, st2 = 0.0;
+            double a1 = 0.0, a2 = 0.0, b1 = 0.0, b2 = 0.0;
             for (int i = 0; i < mine; ++i) {
-                const double xb = (double)key_value(sk[at(j0 + i)]) - centre;
-                const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
-                sb1 += xb; sb2 += xb * xb;
-                st1 += xt; st2 += xt * xt;
+                const uint32_t kb = sk[at(j0 + i)], kt = sk[at(hi0 + j0 + i)];
+                differs |= (kb != kt ? 1u : 0u) << i;
+                const double xb = (double)key_value(kb) - centre;
+                const double xt = (double)key_value(kt) - centre;
+                a1 += xb; a2 += xb * xb;
+                b1 += xt; b2 += xt * xt;
             }
-            double a1, a2, b1, b2;
-            scan(sb1, sb2, st1, st2, a1, a2, b1, b2);
+            scan_both_ends<LANES>(sl, a1, a2, b1, b2);
             for (int i = 0; i < mine; ++i) {
-                consider(j0 + i, a1 + b1, a2 + b2);
+                consider_split<EXACT>(sb, jforce, m, j0 + i, (EXACT ? __popc(differs & ((1u << i) - 1u)) : 0), a1 + b1, a2 + b2);
                 const double xb = (double)key_value(sk[at(j0 + i)]) - centre;
                 const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
                 a1 += xb; a2 += xb * xb;
                 b1 -= xt; b2 -= xt * xt;
             }
-            if (sl == LANES - 1) consider(m, a1, a2);
+            if (sl == LANES - 1) consider_split<EXACT>(sb, jforce, m, m, (EXACT ? __popc(differs) : 0), a1, a2);
         }
+        const double best = sb.best, runner_up = sb.runner_up;
+        const int bestj = sb.j;
+        double bq1 = sb.q1, bq2 = sb.q2;              // sums over the kept subset of my best split
 
         // ---- 4. arg-max over the group: largest score, then largest j --------------------------------------
         int jstar;
@@ -603,6 +743,60 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
             const int owner = owners ? __ffs(owners) - 1 : lane;
             bq1 = __shfl_sync(PODS_FULL_MASK, bq1, owner);
             bq2 = __shfl_sync(PODS_FULL_MASK, bq2, owner);
+            const double best_all = __shfl_sync(PODS_FULL_MASK, best, owner);
+            // Split j+1 swaps the (m-j)-th highest reward for the (j+1)-th lowest; when the two are equal both
+            // splits keep the same multiset of rewards and tie exactly, whatever rounding did to their fp64
+            // scores.  Algorithm 2 keeps the smallest k, i.e. the largest j, of such a run: move up to its end.
+            bool rival = false;
+            if (jforce < 0) {
+                // the run of splits around jstar that keep one and the same multiset
+                auto run_of = [&](int j, int& lo, int& hi, bool want_lo) {
+                    const int from = j - j0;                                  // my positions from here on lie ahead
+                    const uint32_t below = from >= 32 ? 0xffffffffu : (from <= 0 ? 0u : (1u << from) - 1u);
+                    const uint32_t ahead = differs & ~below, behind = differs & below;
+                    const uint32_t stop = ahead != 0u ? (uint32_t)(j0 + __ffs(ahead) - 1) : (uint32_t)m;
+                    hi = max(j, (int)__reduce_min_sync(gmask, stop));
+                    if (want_lo) {
+                        const uint32_t start = behind != 0u ? (uint32_t)(j0 + 32 - __clz(behind)) : 0u;
+                        lo = (int)__reduce_max_sync(gmask, start);
+                    }
+                };
+                int run_lo = 0, run_hi;
+                run_of(jstar, run_lo, run_hi, EXACT);
+                jstar = run_hi;
+                if (EXACT) {
+                    // a rival outside that run whose fp64 score is within 2^-40 of the best: fp64 cannot tell a tie
+                    // from a win there, the exact evaluation has to.  My best if it lies outside the winner's run,
+                    // and my runner-up (outside my best's run, hence outside the winner's whenever my best is inside)
+                    const double near = best_all - fabs(best_all) * 9.094947017729282e-13;
+                    rival = (bestj >= 0 && (bestj < run_lo || bestj > run_hi) && best >= near) || runner_up >= near;
+                    if (c > 4) rival = true;           // long ends (m > 4 LANES): always settled exactly
+                } else if (run_hi >= 1 && run_hi <= m - 1) {
+                    // The one other tie that holds for any values: a kept subset of just two values a < b, j of a and
+                    // m-j of b, scores j (m-j) (b-a)^2, the same as its mirror image (m-j of a, j of b).  fp64 rounds
+                    // the two differently unless the sums are exact; when the mirror image of the run is a split
+                    // too and lies above it, that one is the smaller k.
+                    const uint32_t ka = sk[0], kb2 = sk[at(n - 1)];
+                    const int jm = m - run_hi;                                 // as many of a as there were of b
+                    const bool two_valued = ka != kb2 && sk[at(run_hi - 1)] == ka && (run_hi == m || sk[at(hi0 + run_hi)] == kb2);
+                    const bool mirrored = jm > run_hi && sk[at(jm - 1)] == ka && (jm == m || sk[at(hi0 + jm)] == kb2);
+                    if (two_valued && mirrored) {      // per group; the reductions below use the group's own mask
+                        // the kept sums follow from the counts: x = 0 for a (the minimum), d = b - a for the others
+                        const double d = (double)key_value(kb2) - centre, cntb = (double)run_hi;
+                        run_of(jm, run_lo, run_hi, false);
+                        jstar = run_hi;
+                        bq1 = cntb * d;
+                        bq2 = cntb * d * d;
+                    }
+                }
+            }
+            if (EXACT) {
+                if (__any_sync(PODS_FULL_MASK, rival)) {   // every lane of the warp goes; only the groups concerned listen
+                    double e1, e2;
+                    const int jexact = exact_best_split<LANES, LOGE>(sk, n, m, c, sub, sl, gmask, centre, &e1, &e2);
+                    if (__ballot_sync(PODS_FULL_MASK, rival) & gmask) { jstar = jexact; bq1 = e1; bq2 = e2; }
+                }
+            }
         }
         const int nlo = jstar, nhi = m - jstar;
         const int kstar = nhi;
@@ -731,7 +925,7 @@ int launch_select_fast(const float* rewards, int64_t G, int n, int m, int rule, 
     constexpr int GPW = 32 / LANES;
     // per group: its keys in original and in sorted order, rows of E + 4 words per lane
     const size_t smem = (size_t)kSelectWarps * GPW * 2 * LANES * (E + 4) * sizeof(uint32_t);
-    auto kernel = pods_select_fast_kernel<LANES, E>;
+    auto kernel = (flags & PODS_FLAG_EXACT_TIES) ? pods_select_fast_kernel<LANES, E, true> : pods_select_fast_kernel<LANES, E, false>;
     if (smem > 48 * 1024)
         PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t groups_per_cta = (int64_t)kSelectWarps * GPW;

@@ -54,6 +54,27 @@ def test_every_kernel_shape_and_ragged_n(n):
             _compare(r, m)
 
 
+def test_ties_that_hold_for_any_values_and_ties_by_coincidence():
+    """Splits that keep the same multiset, and the mirror pair of a two-valued kept subset, tie whatever the values
+    are: the default path must get them right for rewards that fp64 sums do not represent exactly.  Ties that hold
+    only because the reward values happen to be commensurate (0.1, 0.2, 0.4 in fp32 are exactly 1 : 2 : 4) are
+    settled exactly under FLAG_EXACT_TIES."""
+    rng = np.random.default_rng(11)
+    for n, m in [(7, 3), (16, 4), (32, 8), (64, 16), (100, 30), (512, 128), (1000, 333)]:
+        for values in ([0.1, 0.7], [0.3, 1.1], [0.1, 0.3, 0.7], [0.0, 0.1, 1.0, 1.1]):
+            r = rng.choice(values, (53, n)).astype(np.float32)
+            _compare(r, m)
+            _compare(r, m, flags=binding.FLAG_EXACT_TIES)
+        base = np.float32(0.1)
+        r = (rng.choice([1.0, 2.0, 4.0], (53, n)).astype(np.float32) * base).astype(np.float32)
+        _compare(r, m, flags=binding.FLAG_EXACT_TIES)
+    # the exact path agrees with the default one where the default is exact by itself
+    for kind, r in _reward_kinds(rng, 67, 48):
+        a = _run(r, 12)
+        b = _run(r, 12, flags=binding.FLAG_EXACT_TIES)
+        assert a[0].tobytes() == b[0].tobytes() and a[2].tobytes() == b[2].tobytes(), kind
+
+
 def test_workload_rewards_at_full_size():
     for name in ("c1_tiny", "c2_qwen_vocab", "c3_select_mixed", "c4_select_ties", "c5_large_loss"):
         w = wl.WORKLOADS[name]
