@@ -48,6 +48,8 @@ typedef enum {
 #define PODS_STATUS_NEG_LENGTH       0x8u  /* pods_compact: a negative length was treated as 0            */
 #define PODS_STATUS_TIMEOUT          0x10u /* a bounded wait inside a kernel ran out (asynchronous copy never
                                               completed); the results of that call are not valid           */
+#define PODS_STATUS_INDEX_RANGE      0x20u /* pods_compact: an entry of idx was outside [0,n); rollout 0 of the
+                                              group was used instead                                        */
 
 /* Down-sampling rules D(o, r; m) of Section 3.2 / 3.3. */
 typedef enum {
@@ -211,7 +213,8 @@ int grpo_loss_chunk_static(const void* logits, int64_t ldl, const int32_t* token
  *   hidden [dev] bf16 [T, d], row pitch ldh elements      W [dev] bf16 [V, d], row pitch ldw elements
  *   tokens [dev] int32 [T] (an id outside [0,V) raises PODS_STATUS_TOKEN_RANGE and is read as 0)
  *   logp   [dev] fp32 [T]                                 lse [dev] fp32 [T] or NULL
- *   workspace [dev] of grpo_logp_from_hidden_workspace_bytes(T, V, d), 16-byte aligned
+ *   workspace [dev] of grpo_logp_from_hidden_workspace_bytes(T, V, d), 16-byte aligned (the size follows from
+ *             the SM count of the device that is current at the query: ask on the device that will run the call)
  * Requires d >= 8 and d % 8 == 0, ldh % 8 == 0, ldw % 8 == 0, 16-byte aligned hidden and W (so that every row
  * starts on a 16-byte boundary); anything else returns PODS_ERR_INVALID_ARG.  Both matrices must live in the
  * current device's own memory.

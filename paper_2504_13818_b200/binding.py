@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libpods_b200.so")
 RULE_MAXVAR, RULE_MAXREWARD, RULE_RANDOM, RULE_PERCENTILE = 0, 1, 2, 3
 FLAG_ADV_BEFORE, FLAG_STD_SAMPLE, FLAG_EXACT_TIES = 1, 2, 4
 STATUS_NONFINITE_REWARD, STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_NEG_LENGTH, STATUS_TIMEOUT = 1, 2, 4, 8, 16
+STATUS_INDEX_RANGE = 32
 MAX_N = 1024
 
 # name -> (restype, argtypes); mirrors include/pods.h

@@ -407,10 +407,9 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 extern "C" size_t grpo_logp_from_hidden_workspace_bytes(int64_t T, int32_t V, int32_t d) {
     (void)d;
     if (T <= 0 || V <= 0) return 0;
-    // the largest number of parts any device's plan can choose is the number of column tiles
-    const size_t tiles = (size_t)((V + BN - 1) / BN);
-    const size_t rows = (size_t)((T + BM - 1) / BM) * BM;
-    return align_up(tiles * rows * sizeof(float2), 256);
+    // one (maximum, sum) pair per row and part of the vocabulary; the parts follow from the current device's SM count
+    const Plan plan = make_plan(T, V, pods_sm_count());
+    return align_up((size_t)plan.n_parts * (size_t)plan.n_row_blocks * BM * sizeof(float2), 256);
 }
 
 extern "C" int grpo_logp_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_t ldw,

@@ -16,6 +16,15 @@ struct StreamPtrs {
     float* dst[kMaxStreams];
 };
 
+// idx[i] as a rollout number of its group: a value outside [0, n) (the caller handed over something that is not
+// pods_select's output) raises PODS_STATUS_INDEX_RANGE and is read as rollout 0, so that no address leaves the storage.
+__device__ __forceinline__ int32_t kept_rollout(const int32_t* idx, int64_t i, int n, uint32_t* status) {
+    const int32_t j = idx[i];
+    if (j >= 0 && j < n) return j;
+    pods_raise(status, PODS_STATUS_INDEX_RANGE);
+    return 0;
+}
+
 // One CTA walks the M kept rollouts in tiles of 1024, carrying the running total: M is the number
 // of kept rollouts of a training batch (hundreds to thousands), far too few to need a
 // multi-CTA scan.
@@ -32,7 +41,7 @@ compact_scan_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__
         int64_t len = 0;
         if (i < M) {
             const int64_t g = i / m;
-            int32_t l = lengths[g * n + idx[i]];
+            int32_t l = lengths[g * n + kept_rollout(idx, i, n, status)];
             if (l < 0) { l = 0; pods_raise(status, PODS_STATUS_NEG_LENGTH); }
             if (l > src_ld) { l = (int32_t)src_ld; pods_raise(status, PODS_STATUS_CAPACITY); }   // longer than its storage row
             len = l;
@@ -73,7 +82,7 @@ compact_gather_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict
                       uint32_t* status) {
     const int64_t i = blockIdx.x;
     const int64_t g = i / m;
-    const int64_t row = g * n + idx[i];
+    const int64_t row = g * n + kept_rollout(idx, i, n, nullptr);     // the scan kernel has raised the bit already
     const int64_t begin = cu_seqlens[i];
     int64_t len = cu_seqlens[i + 1] - begin;
     if (begin + len > T_cap) {

@@ -61,6 +61,26 @@ def test_capacity_and_bad_lengths_raise_status_without_overrun():
     assert int(cu2[1]) == 0
 
 
+def test_kept_indices_outside_the_group_raise_status_and_read_rollout_zero():
+    """idx is data: entries outside [0, n) (not pods_select's output) must not become addresses."""
+    w = wl.WORKLOADS["c1_tiny"]
+    idx, lengths, src, _ = _case(w)
+    bad = idx.copy()
+    bad[1, 2] = w.n                    # one past the group
+    bad[3, 0] = -1000000
+    status = binding.new_status()
+    cu, toks, _ = binding.pods_compact(torch.from_numpy(bad).cuda(), w.n, torch.from_numpy(lengths).cuda(),
+                                       torch.from_numpy(src).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert binding.read_status(status) == binding.STATUS_INDEX_RANGE
+    fixed = bad.copy()
+    fixed[1, 2] = 0
+    fixed[3, 0] = 0
+    cu_o, tok_o, _, _ = oracle.compact(fixed, w.n, lengths, src)
+    np.testing.assert_array_equal(cu.cpu().numpy(), cu_o)
+    np.testing.assert_array_equal(toks[: int(cu_o[-1])].cpu().numpy(), tok_o)
+
+
 def test_seq_weights_with_and_without_mask():
     rng = np.random.default_rng(3)
     lens = rng.integers(0, 70, 50)
