@@ -236,7 +236,7 @@ pods_select_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, i
                     bestk = ok;
                 }
             }
-            kstar = __shfl_sync(PODS_FULL_MASK, bestk, sub * LANES);   // one verdict per group, even with NaN scores
+            kstar = __shfl_sync(PODS_FULL_MASK, bestk, sub * LANES);   // one answer per group, even with NaN scores
             __syncwarp();
         } else if (rule == PODS_RULE_MAXVAR) {
             kstar = 0;                                       // m == n: every split is the whole group

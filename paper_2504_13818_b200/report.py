@@ -2,8 +2,8 @@
 
   python -m paper_2504_13818_b200.report <all_configs.json> <parity_maxima.jsonl>
 
-<all_configs.json> is the line `python bench.py --all-configs` prints; <parity_maxima.jsonl> is what the `-m gpu`
-tests append to (one JSON object per parity case with the maxima they achieved).  Reads the two files and
+<all_configs.json> is the line `python bench.py --all-configs` prints; <parity_maxima.jsonl> is the file the `-m gpu`
+tests append to (PODS_PARITY_RECORD; one JSON object per parity case with the maxima they achieved).  Reads the two files and
 prints; computes nothing of the method."""
 import json
 import sys

@@ -21,12 +21,13 @@ def _built_oracle():
 
 @pytest.fixture(scope="session", autouse=True)
 def _parity_record():
-    """GPU parity tests append the maxima they achieved (not only pass/fail) to gpurun_out/parity_maxima.jsonl."""
+    """GPU parity tests append the maxima they achieved (not only pass/fail) to a JSON-lines record: the file
+    named by PODS_PARITY_RECORD, else parity_maxima.jsonl in pytest's cache folder."""
     import parity
-    out = os.path.join(ROOT, "gpurun_out")
+    path = os.environ.get("PODS_PARITY_RECORD") or os.path.join(ROOT, ".pytest_cache", "parity_maxima.jsonl")
     try:
-        os.makedirs(out, exist_ok=True)
-        parity.RECORD_PATH = os.path.join(out, "parity_maxima.jsonl")
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        parity.RECORD_PATH = path
     except OSError:
         parity.RECORD_PATH = None
     yield

@@ -42,7 +42,7 @@ LOGP_RESOLUTION = 5e-7  # one fp32 ulp of a log-prob in [-8, -4): the grain of t
 # (|x| / ulp(x) < 2^8 for every bf16 x); every other row is held to the literal 2-ulp bound.
 SLACK_ROW_THRESHOLD = 0.25 / 256.0
 
-RECORD_PATH = None      # set by conftest to <repo>/gpurun_out/parity_maxima.jsonl when that folder can be written
+RECORD_PATH = None      # set by conftest: the JSON-lines file the achieved maxima are appended to
 
 
 def record(case, **values):
