@@ -339,12 +339,19 @@ pods_select_kernel(const float* __restrict__ rewards, int64_t G, int n, int m, i
 // reward -> uint32 whose unsigned order is the order of the floats: -0 is folded into +0 by the
 // addition, the sign decides between flipping everything and setting the top bit.  NaNs are dealt
 // with by the caller (they are rare): every NaN gets the key 0xfffffffe, padding 0xffffffff.
-__device__ __forceinline__ uint32_t ordered_key(float r) {
-    const uint32_t u = __float_as_uint(r + 0.0f);
-    return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+// all-ones for a set top bit, 0 otherwise, as the high half of u * 2 (signed): a multiply on the FMA pipe in place
+// of a shift on the integer pipe, which the sort keeps busy (`two` holds an opaque 2)
+__device__ __forceinline__ uint32_t top_bit_mask(uint32_t u, uint32_t two) {
+    uint32_t r;
+    asm("mul.hi.s32 %0, %1, %2;" : "=r"(r) : "r"(u), "r"(two));
+    return r;
 }
-__device__ __forceinline__ float key_value(uint32_t o) {
-    return __uint_as_float(o ^ (~(uint32_t)((int32_t)o >> 31) | 0x80000000u));
+__device__ __forceinline__ uint32_t ordered_key(float r, uint32_t two) {
+    const uint32_t u = __float_as_uint(r + 0.0f);
+    return u ^ (top_bit_mask(u, two) | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(uint32_t o, uint32_t two) {
+    return __uint_as_float(o ^ (~top_bit_mask(o, two) | 0x80000000u));
 }
 
 constexpr uint32_t kKeyNaN = 0xfffffffeu;       // above +inf, below the padding
@@ -493,6 +500,13 @@ __device__ __forceinline__ uint32_t below_mask(uint32_t k, unsigned long long ne
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(k), "r"(one), "l"(neg_v));
     return (uint32_t)(d >> 32);
 }
+// acc <- 2 acc + h with h = 0 or all-ones (-1): fed the elements from the last to the first, -acc ends up as the
+// bit mask of the elements with h = -1 (bit e for element e).  Again a multiply-add (`two` holds an opaque 2).
+__device__ __forceinline__ uint32_t push_mask_bit(uint32_t acc, uint32_t h, uint32_t two) {
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(acc), "r"(two), "r"(h));
+    return r;
+}
 
 // A lane's standing among its own splits: the best score so far with its j and the sums over its kept subset, and
 // the best score among its splits that keep another multiset than that best (`run` numbers the runs of identical
@@ -564,8 +578,9 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
     const int nreal = max(0, min(E, n - sl * E));   // my elements that exist
     const uint32_t real_mask = nreal >= 32 ? 0xffffffffu : ((1u << nreal) - 1u);
     const float pad_value = __uint_as_float(0x7fffffffu);       // its key is kKeyPad
-    uint32_t one;
+    uint32_t one, two;
     asm volatile("mov.u32 %0, 1;" : "=r"(one));
+    asm volatile("mov.u32 %0, 2;" : "=r"(two));
 
     const int64_t stride = (int64_t)gridDim.x * kSelectWarps * GPW;
     for (int64_t base = ((int64_t)blockIdx.x * kSelectWarps + warp) * GPW; base < G; base += stride) {
@@ -581,16 +596,16 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
                 const int i = sl * E + e;
                 float4 v = make_float4(pad_value, pad_value, pad_value, pad_value);
                 if (i < n) v = valid ? *reinterpret_cast<const float4*>(r_g + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                key[e] = ordered_key(v.x);
-                key[e + 1] = ordered_key(v.y);
-                key[e + 2] = ordered_key(v.z);
-                key[e + 3] = ordered_key(v.w);
+                key[e] = ordered_key(v.x, two);
+                key[e + 1] = ordered_key(v.y, two);
+                key[e + 2] = ordered_key(v.z, two);
+                key[e + 3] = ordered_key(v.w, two);
             }
         } else {
 #pragma unroll
             for (int e = 0; e < E; ++e) {
                 const int i = sl * E + e;
-                key[e] = ordered_key(i < n ? (valid ? r_g[i] : 0.0f) : pad_value);
+                key[e] = ordered_key(i < n ? (valid ? r_g[i] : 0.0f) : pad_value, two);
             }
         }
 #pragma unroll
@@ -669,7 +684,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         // ---- 3. fp64 running sums of the centred rewards over the two ends of the sorted order ------------
         const bool nonfinite = k_min <= kKeyNegInf || k_max >= kKeyPosInf;
         if (nonfinite && valid && sl == 0) pods_raise(status, PODS_STATUS_NONFINITE_REWARD);
-        const double centre = (double)key_value(k_min);                      // the group minimum
+        const double centre = (double)key_value(k_min, two);                      // the group minimum
         const int j0 = sl * c;                                               // my splits: j0 .. j0 + mine - 1
         const int mine = max(0, min(c, m - j0));
         const int hi0 = n - m;                        // sorted position j is the j-th lowest, hi0 + j the (m-j)-th highest
@@ -689,8 +704,8 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
                 if (i < mine) {
                     const uint32_t kb = sk[at(j0 + i)], kt = sk[at(hi0 + j0 + i)];
                     differs |= (kb != kt ? 1u : 0u) << i;
-                    xb[i] = (double)key_value(kb) - centre;
-                    xt[i] = (double)key_value(kt) - centre;
+                    xb[i] = (double)key_value(kb, two) - centre;
+                    xt[i] = (double)key_value(kt, two) - centre;
                 }
                 a1 += xb[i]; a2 += xb[i] * xb[i];
                 b1 += xt[i]; b2 += xt[i] * xt[i];
@@ -709,16 +724,16 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
             for (int i = 0; i < mine; ++i) {
                 const uint32_t kb = sk[at(j0 + i)], kt = sk[at(hi0 + j0 + i)];
                 differs |= (kb != kt ? 1u : 0u) << i;
-                const double xb = (double)key_value(kb) - centre;
-                const double xt = (double)key_value(kt) - centre;
+                const double xb = (double)key_value(kb, two) - centre;
+                const double xt = (double)key_value(kt, two) - centre;
                 a1 += xb; a2 += xb * xb;
                 b1 += xt; b2 += xt * xt;
             }
             scan_both_ends<LANES>(sl, a1, a2, b1, b2);
             for (int i = 0; i < mine; ++i) {
                 consider_split<EXACT>(sb, jforce, m, j0 + i, (EXACT ? __popc(differs & ((1u << i) - 1u)) : 0), a1 + b1, a2 + b2);
-                const double xb = (double)key_value(sk[at(j0 + i)]) - centre;
-                const double xt = (double)key_value(sk[at(hi0 + j0 + i)]) - centre;
+                const double xb = (double)key_value(sk[at(j0 + i)], two) - centre;
+                const double xt = (double)key_value(sk[at(hi0 + j0 + i)], two) - centre;
                 a1 += xb; a2 += xb * xb;
                 b1 -= xt; b2 -= xt * xt;
             }
@@ -782,7 +797,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
                     const bool mirrored = jm > run_hi && sk[at(jm - 1)] == ka && (jm == m || sk[at(hi0 + jm)] == kb2);
                     if (two_valued && mirrored) {      // per group; the reductions below use the group's own mask
                         // the kept sums follow from the counts: x = 0 for a (the minimum), d = b - a for the others
-                        const double d = (double)key_value(kb2) - centre, cntb = (double)run_hi;
+                        const double d = (double)key_value(kb2, two) - centre, cntb = (double)run_hi;
                         run_of(jm, run_lo, run_hi, false);
                         jstar = run_hi;
                         bq1 = cntb * d;
@@ -808,7 +823,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
 #pragma unroll 4
             for (int e = 0; e < E; ++e) {
                 if (e < nreal) {
-                    const double x = (double)key_value(sk[sl * ROWW + e]) - centre;
+                    const double x = (double)key_value(sk[sl * ROWW + e], two) - centre;
                     f1 += x; f2 += x * x;
                 }
             }
@@ -830,32 +845,36 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         uint32_t take = 0u;
         if (!__any_sync(PODS_FULL_MASK, cut)) {
             // no run is cut anywhere in the warp: everything up to v_lo and everything from v_hi on is kept
+            const unsigned long long neg_le = 0ull - (unsigned long long)v_lo - 1ull, neg_hi = 0ull - (unsigned long long)v_hi;
+            uint32_t a_le = 0u, a_lth = 0u;                     // minus the masks "up to v_lo" and "below v_hi"
 #pragma unroll
-            for (int e = 0; e < E; e += 4) {
+            for (int e = E - 4; e >= 0; e -= 4) {
                 const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
                 const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-                for (int t = 0; t < 4; ++t) take |= ((kk[t] <= v_lo || kk[t] >= v_hi) ? 1u : 0u) << (e + t);
+                for (int t = 3; t >= 0; --t) {
+                    a_le = push_mask_bit(a_le, below_mask(kk[t], neg_le, one), two);
+                    a_lth = push_mask_bit(a_lth, below_mask(kk[t], neg_hi, one), two);
+                }
             }
-            take &= real_mask;
+            take = ((0u - a_le) | ~(0u - a_lth)) & real_mask;
         } else {
-            // four masks over my rewards: below v_lo, up to v_lo, below v_hi, up to v_hi
+            // four masks over my rewards: below v_lo, up to v_lo, below v_hi, up to v_hi (all on the FMA pipe)
             const unsigned long long neg_lo = 0ull - (unsigned long long)v_lo, neg_hi = 0ull - (unsigned long long)v_hi;
             uint32_t m_lt = 0u, m_le = 0u, m_lth = 0u, m_leh = 0u;
 #pragma unroll
-            for (int e = 0; e < E; e += 4) {
+            for (int e = E - 4; e >= 0; e -= 4) {
                 const uint4 q = *reinterpret_cast<const uint4*>(ok + sl * ROWW + e);
                 const uint32_t kk[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const uint32_t bit = 1u << (e + t);
-                    m_lt |= below_mask(kk[t], neg_lo, one) & bit;
-                    m_le |= below_mask(kk[t], neg_lo - 1ull, one) & bit;
-                    m_lth |= below_mask(kk[t], neg_hi, one) & bit;
-                    m_leh |= below_mask(kk[t], neg_hi - 1ull, one) & bit;
+                for (int t = 3; t >= 0; --t) {
+                    m_lt = push_mask_bit(m_lt, below_mask(kk[t], neg_lo, one), two);
+                    m_le = push_mask_bit(m_le, below_mask(kk[t], neg_lo - 1ull, one), two);
+                    m_lth = push_mask_bit(m_lth, below_mask(kk[t], neg_hi, one), two);
+                    m_leh = push_mask_bit(m_leh, below_mask(kk[t], neg_hi - 1ull, one), two);
                 }
             }
-            m_lt &= real_mask;
+            m_lt = (0u - m_lt) & real_mask; m_le = 0u - m_le; m_lth = 0u - m_lth; m_leh = 0u - m_leh;
             const uint32_t m_el = m_le & ~m_lt & real_mask;              // equal to v_lo
             const uint32_t m_gt = ~m_leh & real_mask;                    // above v_hi
             const uint32_t m_eh = m_leh & ~m_lth & real_mask;            // equal to v_hi
@@ -909,7 +928,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
             float* ao = adv_out + g * (int64_t)m;
             for (int j = sl; j < m; j += LANES) {
                 const int i = stage[j] & (NPAD - 1);
-                const double xi = (double)key_value(ok[at(i)]) - centre;
+                const double xi = (double)key_value(ok[at(i)], two) - centre;
                 io[j] = i;
                 ao[j] = (float)((xi * cnt - s1) * inv_sigma_c);
             }
