@@ -48,6 +48,8 @@ typedef enum {
 #define PODS_STATUS_NEG_LENGTH       0x8u  /* pods_compact: a negative length was treated as 0            */
 #define PODS_STATUS_TIMEOUT          0x10u /* a bounded wait inside a kernel ran out (asynchronous copy never
                                               completed); the results of that call are not valid           */
+#define PODS_STATUS_INTERNAL         0x40u /* checked build only (-DPODS_BOUNDS_CHECK): an index computed inside a
+                                              kernel left its extent; the access was skipped               */
 #define PODS_STATUS_INDEX_RANGE      0x20u /* pods_compact: an entry of idx was outside [0,n); rollout 0 of the
                                               group was used instead                                        */
 

@@ -12,12 +12,13 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpods_b200.so")
+# PODS_B200_LIBRARY names another build of the same library (the tests load the checked build through it)
+LIB_PATH = os.environ.get("PODS_B200_LIBRARY") or os.path.join(_HERE, "libpods_b200.so")
 
 RULE_MAXVAR, RULE_MAXREWARD, RULE_RANDOM, RULE_PERCENTILE = 0, 1, 2, 3
 FLAG_ADV_BEFORE, FLAG_STD_SAMPLE, FLAG_EXACT_TIES = 1, 2, 4
 STATUS_NONFINITE_REWARD, STATUS_TOKEN_RANGE, STATUS_CAPACITY, STATUS_NEG_LENGTH, STATUS_TIMEOUT = 1, 2, 4, 8, 16
-STATUS_INDEX_RANGE = 32
+STATUS_INDEX_RANGE, STATUS_INTERNAL = 32, 64
 MAX_N = 1024
 
 # name -> (restype, argtypes); mirrors include/pods.h

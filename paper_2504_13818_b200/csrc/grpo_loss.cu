@@ -259,7 +259,7 @@ grpo_loss_rows_kernel(const RowArgs a) {
 #pragma unroll
                 for (int j = 0; j < kBatch; ++j) {
                     const int v = v0 + j * BLOCK;
-                    if (v < nvec) {
+                    if (v < nvec && PODS_INDEX_OK((int64_t)v * 8 + 7, a.ldd, a.status)) {
                         uint4 o = grad_vec(q[j], coef, ref);
                         if (v == tok_vec) patch_bf16(o, tok & 7, target_bits);
                         __stcs(d4 + v, o);
@@ -363,7 +363,7 @@ grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
                 const float part = (k == excl) ? exp_sum_excluding(q[k], ref, mx) : 0.0f;
                 const float sum = exp_vec_inplace(q[k], ref);
                 if (k & 1) s1 += (k == excl) ? part : sum; else s0 += (k == excl) ? part : sum;
-                if (j < nvec) tile[(size_t)r * nvec + j] = q[k];
+                if (j < nvec && PODS_INDEX_OK((size_t)r * nvec + j, (size_t)rows_per_tile * nvec, a.status)) tile[(size_t)r * nvec + j] = q[k];
             }
             float sw = s0 + s1;
 #pragma unroll
@@ -407,7 +407,8 @@ grpo_loss_tile_kernel(const RowArgs a, const int rows_per_tile) {
 #pragma unroll
             for (int k = 0; k < IT; ++k) {
                 const int j = lane + 32 * k;
-                if (j < nvec) {
+                if (j < nvec && PODS_INDEX_OK((size_t)r * nvec + j, (size_t)rows_per_tile * nvec, a.status) &&
+                    PODS_INDEX_OK(tile0 + r, a.T, a.status)) {
                     uint4 e = tile[(size_t)r * nvec + j];
                     scale_vec(e, c_hi, c_lo);
                     out[j] = e;

@@ -408,7 +408,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 for (int k = 0; k < IT; ++k) {
                     const int j = lo + lane + 32 * k;
                     scale_vec(q[k], c_hi, c_lo);
-                    if (j < hi) out[j] = q[k];
+                    if (j < hi && PODS_INDEX_OK(seg0 + j, nvec, a.status) && PODS_INDEX_OK(t, a.T, a.status)) out[j] = q[k];
                 }
                 // the target entry, if it is in my slice: rewritten by the lane that stored its vector
                 if (tok_vec >= lo && tok_vec < hi && ((tok_vec - lo) & 31) == lane)
@@ -463,7 +463,7 @@ grpo_loss_cluster_kernel(const RowArgs a, const int seg_vecs, const int n_stages
                 const float part = (k == excl) ? exp_sum_excluding(q[k], ref_w, m_w) : 0.0f;
                 const float sum = exp_vec_inplace(q[k], ref_w);
                 if (k & 1) s1 += (k == excl) ? part : sum; else s0 += (k == excl) ? part : sum;
-                if (j < hi) buf[j] = q[k];
+                if (j < hi && PODS_INDEX_OK(j, stage_vecs, a.status)) buf[j] = q[k];
             }
             float sw = s0 + s1;
 #pragma unroll

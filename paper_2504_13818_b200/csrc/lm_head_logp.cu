@@ -280,7 +280,8 @@ lm_head_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __gri
                 if (lane == 0) mbar_arrive(&bar.acc_empty[acc]);
                 if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
             }
-            a.partial[(size_t)part * ((size_t)a.n_row_blocks * BM) + (size_t)rb * BM + row_in_tile] = make_float2(m_run, s_run);
+            const size_t slot = (size_t)part * ((size_t)a.n_row_blocks * BM) + (size_t)rb * BM + row_in_tile;
+            if (PODS_INDEX_OK(slot, (size_t)a.n_parts * a.n_row_blocks * BM, a.status)) a.partial[slot] = make_float2(m_run, s_run);
         }
     }
     if (timed_out && lane == 0) pods_raise(a.status, PODS_STATUS_TIMEOUT);

@@ -31,3 +31,22 @@ static inline int pods_sm_count() {
 __device__ __forceinline__ void pods_raise(uint32_t* status, uint32_t bit) {
     if (status != nullptr) atomicOr(status, bit);
 }
+
+// Checked build (-DPODS_BOUNDS_CHECK, a separate library used by the tests in place of a memory checker): an index
+// that the kernels compute is compared with the extent it must stay inside; a violation ORs PODS_STATUS_INTERNAL
+// into the status word and the access is skipped - never a trap.  In the normal build the test is the constant
+// true and costs nothing.
+#ifdef PODS_BOUNDS_CHECK
+__device__ __forceinline__ bool pods_index_ok(long long i, long long extent, uint32_t* status) {
+    if (i >= 0 && i < extent) return true;
+    pods_raise(status, PODS_STATUS_INTERNAL);
+    return false;
+}
+#define PODS_INDEX_OK(i, extent, status) pods_index_ok((long long)(i), (long long)(extent), (status))
+// the index itself if it is inside its extent, else 0 (with the bit raised): for loads whose value feeds warp-wide
+// operations, where skipping is not an option
+#define PODS_CLAMPED(i, extent, status) (pods_index_ok((long long)(i), (long long)(extent), (status)) ? (i) : 0)
+#else
+#define PODS_INDEX_OK(i, extent, status) true
+#define PODS_CLAMPED(i, extent, status) (i)
+#endif

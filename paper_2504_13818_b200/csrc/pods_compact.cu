@@ -90,11 +90,13 @@ compact_gather_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict
         len = T_cap > begin ? T_cap - begin : 0;
     }
     const int32_t* st = src_tokens + row * src_ld;
-    for (int64_t t = threadIdx.x; t < len; t += blockDim.x) dst_tokens[begin + t] = st[t];
+    for (int64_t t = threadIdx.x; t < len; t += blockDim.x)
+        if (PODS_INDEX_OK(begin + t, T_cap, status) && PODS_INDEX_OK(t, src_ld, status)) dst_tokens[begin + t] = st[t];
     for (int s = 0; s < n_f32; ++s) {
         const float* sp = streams.src[s] + row * src_ld;
         float* dp = streams.dst[s] + begin;
-        for (int64_t t = threadIdx.x; t < len; t += blockDim.x) dp[t] = sp[t];
+        for (int64_t t = threadIdx.x; t < len; t += blockDim.x)
+            if (PODS_INDEX_OK(begin + t, T_cap, status) && PODS_INDEX_OK(t, src_ld, status)) dp[t] = sp[t];
     }
     (void)lengths;
 }

@@ -702,7 +702,8 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
             for (int i = 0; i < 4; ++i) {
                 xb[i] = 0.0; xt[i] = 0.0;
                 if (i < mine) {
-                    const uint32_t kb = sk[at(j0 + i)], kt = sk[at(hi0 + j0 + i)];
+                    const uint32_t kb = sk[PODS_CLAMPED(at(j0 + i), GROUPW, status)];
+                    const uint32_t kt = sk[PODS_CLAMPED(at(PODS_CLAMPED(hi0 + j0 + i, n, status)), GROUPW, status)];
                     differs |= (kb != kt ? 1u : 0u) << i;
                     xb[i] = (double)key_value(kb, two) - centre;
                     xt[i] = (double)key_value(kt, two) - centre;
@@ -837,8 +838,8 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
 
         // ---- 5. the two thresholds; my rewards in original order against them ---------------------------
         // keys of real rewards lie in [1, 0xfffffffe]: 0 and 0xffffffff match nothing when an end is empty
-        const uint32_t v_lo = nlo > 0 ? sk[at(nlo - 1)] : 0u;
-        const uint32_t v_hi = nhi > 0 ? sk[at(n - nhi)] : kKeyPad;
+        const uint32_t v_lo = nlo > 0 ? sk[at(PODS_CLAMPED(nlo - 1, n, status))] : 0u;
+        const uint32_t v_hi = nhi > 0 ? sk[at(PODS_CLAMPED(n - nhi, n, status))] : kKeyPad;
         // a run of equal rewards is cut when the sorted neighbour just outside a kept end has the end's value
         const bool cut = (nlo > 0 && nlo < n && sk[at(nlo)] == v_lo) || (nhi > 0 && nhi < n && sk[at(n - nhi - 1)] == v_hi);
         __syncwarp();                                    // sk has been read for the last time: it becomes `stage`
@@ -914,7 +915,7 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
         off -= my_takes;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if ((take >> e) & 1u) stage[off++] = sl * E + e;
+            if (((take >> e) & 1u) && PODS_INDEX_OK(off, m, status)) stage[off++] = sl * E + e;
         }
         __syncwarp();
 
@@ -928,9 +929,11 @@ pods_select_fast_kernel(const float* __restrict__ rewards, int64_t G, int n, int
             float* ao = adv_out + g * (int64_t)m;
             for (int j = sl; j < m; j += LANES) {
                 const int i = stage[j] & (NPAD - 1);
-                const double xi = (double)key_value(ok[at(i)], two) - centre;
-                io[j] = i;
-                ao[j] = (float)((xi * cnt - s1) * inv_sigma_c);
+                const double xi = (double)key_value(ok[at(PODS_CLAMPED(i, n, status))], two) - centre;
+                if (PODS_INDEX_OK(stage[j], n, status) && PODS_INDEX_OK(g * (int64_t)m + j, G * (int64_t)m, status)) {
+                    io[j] = i;
+                    ao[j] = (float)((xi * cnt - s1) * inv_sigma_c);
+                }
             }
             if (sl == 0 && k_out != nullptr) k_out[g] = kstar;
         }
