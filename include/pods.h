@@ -227,6 +227,49 @@ int grpo_logp_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_
                           size_t workspace_bytes, uint32_t* status, void* stream);
 
 /*
+ * grpo_loss_from_hidden - the token terms of L_PODS(theta, S) (Section 3.2) for rows [row0, row0 + T) of the packed
+ * kept tokens when the logits are the LM-head projection of the last hidden states, together with the gradient
+ * carried back through that projection; neither the [T,V] logits nor their gradient is ever stored in full:
+ *   logits[t, :] = hidden[t, :] . W^T  (bf16 inputs, fp32 accumulation on the tensor cores, not rounded to bf16)
+ *   logp, loss_t, g_t as in grpo_loss_chunk;   dlogits[t, v] = g_t ([v == token] - softmax(logits[t, :])[v])
+ *   dhidden[t, :]  = sum_v dlogits[t, v] W[v, :]           (written: fp32 [T, d], row pitch lddh elements)
+ *   dW[v, :]      += sum_t dlogits[t, v] hidden[t, :]      (ADDED to fp32 [V, d], row pitch lddw elements: the
+ *                                                           caller zeroes it before the first chunk of a batch)
+ * and sum_t mask_t w_i loss_t is ADDED to *loss_acc.  dlogits is rounded to bf16 (nearest even) before it is
+ * contracted, as the gradient grpo_loss_chunk writes is; it exists only one panel of the vocabulary at a time,
+ * inside the workspace (at most 512 MB, whatever T and V).  The logits are formed twice (once for the row
+ * statistics, once for the gradient): the second pass is the price of not storing them.
+ * This is the gradient half of fusing the LM-head projection into the objective; grpo_logp_from_hidden is the
+ * half for passes that need no gradient.
+ *
+ *   hidden [dev] bf16 [T, d] pitch ldh; W [dev] bf16 [V, d] pitch ldw (d >= 8, d % 8 == 0, ldh % 8 == 0,
+ *          ldw % 8 == 0, 16-byte aligned bases), both in the current device's own memory
+ *   tokens, old_logp, ref_logp (NULL allowed iff beta == 0), mask (NULL = all ones), logp (out): [dev] arrays of T
+ *   adv [dev] fp32 [M]; seq_weight [dev] fp64 [M]; cu_seqlens [dev] int64 [M+1]; row0: first packed row of the chunk
+ *   dhidden, dW: [dev] fp32, 16-byte aligned, lddh % 4 == 0, lddw % 4 == 0; they must not overlap anything else
+ *   loss_acc [dev] fp64 scalar; workspace [dev] of grpo_loss_from_hidden_workspace_bytes(T, V, d), 256-byte
+ *   aligned (the size follows from the SM count of the current device: ask on the device that runs the call)
+ * A token id outside [0,V) raises PODS_STATUS_TOKEN_RANGE and is read as 0; a wait that runs out raises
+ * PODS_STATUS_TIMEOUT.  Invalid sizes or pointers return PODS_ERR_INVALID_ARG before anything is launched.
+ */
+size_t grpo_loss_from_hidden_workspace_bytes(int64_t T, int32_t V, int32_t d);
+int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_t ldw, const int32_t* tokens,
+                          const float* old_logp, const float* ref_logp, const float* adv, const double* seq_weight,
+                          const int64_t* cu_seqlens, int64_t M, int64_t row0, const uint8_t* mask, int64_t T,
+                          int32_t V, int32_t d, float eps, float beta, float grad_scale, double* loss_acc,
+                          float* logp, float* dhidden, int64_t lddh, float* dW, int64_t lddw, void* workspace,
+                          size_t workspace_bytes, uint32_t* status, void* stream);
+
+/*
+ * pods_set_loss_from_hidden_panel_bytes - tuning knob (the paper has no counterpart): the most bytes of workspace
+ * grpo_loss_from_hidden may spend on the piece of the logits gradient that exists at one time (default 512 MB; at
+ * least one 256-column tile per panel is always taken; values below 64 KB are raised to 64 KB).  Smaller panels
+ * mean less memory and more passes over dhidden.  Process-wide; changes what grpo_loss_from_hidden_workspace_bytes
+ * returns; returns the previous value.  Results meet the same tolerances at any setting.
+ */
+size_t pods_set_loss_from_hidden_panel_bytes(size_t bytes);
+
+/*
  * pods_set_loss_cluster_min_vocab - tuning knob (the paper has no counterpart): grpo_loss_chunk runs rows of
  * V >= min_vocab (V % 8 == 0, 16-byte aligned rows) on the cluster-resident kernel and shorter rows on the
  * row-tile (V <= 4096) or the general row kernel.  The default, 8192, is the measured cross-over on B200; values

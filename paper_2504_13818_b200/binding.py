@@ -43,6 +43,10 @@ SIGNATURES = {
     "grpo_loss_finalize": (C.c_int, [_p, _p, _p]),
     "grpo_logp_from_hidden_workspace_bytes": (_sz, [_i64, _i32, _i32]),
     "grpo_logp_from_hidden": (C.c_int, [_p, _i64, _p, _i64, _p, _i64, _i32, _i32, _p, _p, _p, _sz, _p, _p]),
+    "grpo_loss_from_hidden_workspace_bytes": (_sz, [_i64, _i32, _i32]),
+    "pods_set_loss_from_hidden_panel_bytes": (_sz, [_sz]),
+    "grpo_loss_from_hidden": (C.c_int, [_p, _i64, _p, _i64, _p, _p, _p, _p, _p, _p, _i64, _i64, _p, _i64, _i32, _i32,
+                                        _f32, _f32, _f32, _p, _p, _p, _i64, _p, _i64, _p, _sz, _p, _p]),
     "pods_selftest_bounded_wait": (C.c_int, [_u32, _p, _p]),
     "pods_set_loss_cluster_min_vocab": (_i32, [_i32]),
     "pods_host_step_create": (C.c_int, [_i64, _i32, _i32, _i64, _i64, _i32, _i64, _p]),
@@ -370,6 +374,67 @@ def grpo_logp_from_hidden(hidden, W, tokens, logp=None, lse=None, want_lse=False
                                       _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "grpo_logp_from_hidden")
     return logp, lse
+
+
+def grpo_loss_from_hidden_workspace_bytes(T, V, d) -> int:
+    return int(load().grpo_loss_from_hidden_workspace_bytes(T, V, d))
+
+
+def set_loss_from_hidden_panel_bytes(nbytes) -> int:
+    """Limit of the gradient panel grpo_loss_from_hidden keeps in its workspace; returns the previous setting."""
+    return int(load().pods_set_loss_from_hidden_panel_bytes(int(nbytes)))
+
+
+def _f32_rows(t, rows, cols, name):
+    """Pointer and row pitch of a 2-D fp32 CUDA tensor [rows, cols] whose rows are contiguous."""
+    _require(isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.dim() == 2 and
+             tuple(t.shape) == (rows, cols) and t.stride(1) == 1,
+             "%s must be a CUDA float32 tensor [%d, %d] with contiguous rows" % (name, rows, cols))
+    return C.c_void_p(t.data_ptr()), (t.stride(0) if rows > 1 else max(t.stride(0), cols))
+
+
+def grpo_loss_from_hidden(hidden, W, tokens, old_logp, ref_logp, adv, seq_weight, cu_seqlens, row0, mask, eps, beta,
+                          loss_acc, dW, logp=None, dhidden=None, workspace=None, grad_scale=1.0, status=None):
+    """Rows [row0, row0+T) of the objective on logits = hidden W^T, with dhidden (written) and dW (added to).
+
+    hidden [T,d] bf16, W [V,d] bf16; loss_acc [1] fp64 and dW [V,d] fp32 accumulate (the caller zeroes them before
+    the first chunk).  Returns (logp [T] fp32, dhidden [T,d] fp32); missing ones and the workspace are allocated here."""
+    _require(isinstance(hidden, torch.Tensor) and hidden.dim() == 2 and isinstance(W, torch.Tensor) and W.dim() == 2,
+             "hidden must be [T,d] and W [V,d]")
+    T, d = hidden.shape
+    V = W.shape[0]
+    _require(W.shape[1] == d, "W must have d = %d columns, got %d" % (d, W.shape[1]))
+    M = cu_seqlens.shape[0] - 1
+    dev = hidden.device
+    if logp is None:
+        logp = torch.empty(T, dtype=torch.float32, device=dev)
+    if dhidden is None:
+        dhidden = torch.empty((T, d), dtype=torch.float32, device=dev)
+    for t, name in ((tokens, "tokens"), (old_logp, "old_logp"), (ref_logp, "ref_logp"), (mask, "mask"), (logp, "logp")):
+        _numel(t, T, name)
+    _numel(adv, M, "adv")
+    _numel(seq_weight, M, "seq_weight")
+    _numel(loss_acc, 1, "loss_acc")
+    need = grpo_loss_from_hidden_workspace_bytes(T, V, d)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    _require(workspace.numel() >= need, "workspace must hold %d bytes, got %d" % (need, workspace.numel()))
+    hp, ldh = _rows(hidden, "hidden")
+    wp, ldw = _rows(W, "W")
+    dhp, lddh = _f32_rows(dhidden, T, d, "dhidden")
+    dwp, lddw = _f32_rows(dW, V, d, "dW")
+    rc = load().grpo_loss_from_hidden(hp, ldh, wp, ldw, _dev(tokens, torch.int32, "tokens"),
+                                      _dev(old_logp, torch.float32, "old_logp"),
+                                      _dev(ref_logp, torch.float32, "ref_logp", True),
+                                      _dev(adv.reshape(-1), torch.float32, "adv"),
+                                      _dev(seq_weight, torch.float64, "seq_weight"),
+                                      _dev(cu_seqlens, torch.int64, "cu_seqlens"), M, row0,
+                                      _dev(mask, torch.uint8, "mask", True), T, V, d, eps, beta, grad_scale,
+                                      _dev(loss_acc, torch.float64, "loss_acc"), _dev(logp, torch.float32, "logp"),
+                                      dhp, lddh, dwp, lddw, _dev(workspace, torch.uint8, "workspace"),
+                                      workspace.numel(), _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "grpo_loss_from_hidden")
+    return logp, dhidden
 
 
 class HostStep:

@@ -465,6 +465,12 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
+int pods_loss::launch_loss_reduce(const double* row_loss, int64_t T, double* loss_acc, cudaStream_t stream) {
+    loss_reduce_kernel<<<1, 1024, 0, stream>>>(row_loss, T, loss_acc);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
 extern "C" size_t grpo_loss_chunk_workspace_bytes(int64_t T_chunk) {
     if (T_chunk < 0) return 0;
     return align_up((size_t)T_chunk * sizeof(double), 256) + align_up((size_t)T_chunk * sizeof(RowPrep), 256) + 256;

@@ -221,9 +221,34 @@ __device__ __forceinline__ RowInputs load_row_inputs(const RowArgs& a, int64_t t
     return in;
 }
 
-// The scalar part of the objective for one token (Section 3.2), fp64:
-//   logp = (x_tok - M) - log(1 + Z'),  rho = exp(logp - old),  loss = -min(rho a, clip(rho) a) + beta kl,
-//   g = grad_scale w dloss/dlogp,  1 - p accurate even when p -> 1.
+// The token term of the objective (Section 3.2) from the token's log-prob, fp64:
+//   rho = exp(logp - old),  loss = -min(rho a, clip(rho) a) + beta kl,  g = grad_scale w dloss/dlogp.
+struct TokenTerms {
+    double weighted_loss, g;
+};
+
+__device__ __forceinline__ TokenTerms token_terms(double logp, const RowInputs& in, float eps_f, float beta_f,
+                                                  float grad_scale) {
+    TokenTerms r;
+    const double eps = (double)eps_f, beta = (double)beta_f;
+    const double rho = exp(logp - in.old_logp);
+    const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
+    const double s1 = rho * in.adv, s2 = clipped * in.adv;
+    double loss = -(s1 < s2 ? s1 : s2);
+    double dl = (s1 <= s2) ? -in.adv * rho : 0.0;
+    if (in.has_ref) {
+        const double d = in.ref_logp - logp;
+        const double ed = exp(d);
+        loss += beta * (ed - d - 1.0);
+        dl += beta * (1.0 - ed);
+    }
+    r.g = (in.w != 0.0) ? (double)grad_scale * in.w * dl : 0.0;
+    r.weighted_loss = (in.w != 0.0) ? in.w * loss : 0.0;     // a masked row adds nothing, whatever its inputs
+    return r;
+}
+
+// The scalar part of the objective for one row of logits:
+//   logp = (x_tok - M) - log(1 + Z'),  the token's terms,  1 - p accurate even when p -> 1.
 struct RowScalars {
     double logp, weighted_loss, g, one_minus_p, Z;
 };
@@ -233,23 +258,15 @@ __device__ __forceinline__ RowScalars row_scalars(const RowArgs& a, const RowInp
     RowScalars r;
     r.Z = 1.0 + zp;
     r.logp = ((double)x_tok - (double)mx) - log1p(zp);
-    const double eps = (double)a.eps, beta = (double)a.beta;
-    const double rho = exp(r.logp - in.old_logp);
-    const double clipped = rho < 1.0 - eps ? 1.0 - eps : (rho > 1.0 + eps ? 1.0 + eps : rho);
-    const double s1 = rho * in.adv, s2 = clipped * in.adv;
-    double loss = -(s1 < s2 ? s1 : s2);
-    double dl = (s1 <= s2) ? -in.adv * rho : 0.0;
-    if (in.has_ref) {
-        const double d = in.ref_logp - r.logp;
-        const double ed = exp(d);
-        loss += beta * (ed - d - 1.0);
-        dl += beta * (1.0 - ed);
-    }
-    r.g = (in.w != 0.0) ? (double)a.grad_scale * in.w * dl : 0.0;
-    r.weighted_loss = (in.w != 0.0) ? in.w * loss : 0.0;     // a masked row adds nothing, whatever its inputs
+    const TokenTerms tt = token_terms(r.logp, in, a.eps, a.beta, a.grad_scale);
+    r.g = tt.g;
+    r.weighted_loss = tt.weighted_loss;
     r.one_minus_p = (x_tok == mx) ? zp / r.Z : -expm1(r.logp);
     return r;
 }
+
+// grpo_loss.cu: fixed-order sum of per-row loss terms, added to *loss_acc (one CTA).
+int launch_loss_reduce(const double* row_loss, int64_t T, double* loss_acc, cudaStream_t stream);
 
 // grpo_loss_cluster.cu: runs the rows on the cluster-resident path when their shape allows it.
 int launch_grpo_loss_cluster(const RowArgs& a, cudaStream_t stream, bool* launched);

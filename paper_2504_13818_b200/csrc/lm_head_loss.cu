@@ -1,0 +1,547 @@
+// grpo_loss_from_hidden: L_PODS (Section 3.2) and its gradient when the logits are the LM-head projection
+// hidden W^T, with the [T,V] logits and their gradient never stored in full: the gradient goes straight on to
+// d loss / d hidden and d loss / d W.
+//
+// Per call (T rows of one chunk):
+//   1. statistics pass (lm_head_logp.cu): logits tile by tile on the tensor cores -> per-row log-sum-exp;
+//   2. lm_head_row_terms_kernel: log-prob, the token's loss term and its gradient factor g_t (fp64 scalars);
+//   then, for one panel of the vocabulary after the other (a panel is as many 256-column tiles as keep the
+//   panel's gradient block within a byte limit, 512 MB unless changed):
+//   3. lm_head_dlogits_kernel: the panel's logits AGAIN on the tensor cores (same pipeline as pass 1), and in the
+//      epilogue dlogits = g_t ([v == token] - 2^(x log2e - lse log2e)) rounded to bf16 into the panel buffer
+//      [rows, panel columns] - the only place a piece of the [T,V] gradient ever exists;
+//   4. lm_head_grad_gemm_kernel<false>: dhidden[T,d] (+)= panel[T, cols] . W[cols, d]
+//   5. lm_head_grad_gemm_kernel<true>:  dW[cols, d] += panel^T[cols, T] . hidden[T, d]
+//      both with tcgen05.mma reading the operands whose contraction index is NOT contiguous in memory (W and hidden
+//      by rows of d, the panel by rows of vocabulary entries for step 5) as MN-major shared-memory tiles, so
+//      no transposed copy of anything is made.
+// Roles, barriers and bounded waits are those of the statistics kernel: a TMA producer warp, one thread issuing
+// the MMAs into one of two 256-column accumulators in tensor memory, four epilogue warps (one tile row per
+// thread).  All loads are plain (never multicast) TMA loads of this GPU's own memory.
+
+#include "grpo_loss_common.cuh"
+#include "lm_head_common.cuh"
+
+using namespace pods_lm;
+
+namespace {
+
+// Upper limit of the gradient panel (rows x panel columns, bf16); pods_set_loss_from_hidden_panel_bytes moves it.
+size_t g_panel_bytes = (size_t)512 << 20;
+
+// What the gradient epilogue needs of a row: 16 bytes.
+struct __align__(16) RowGrad {
+    float g;             // grad_scale mask_t w_i dloss/dlogp
+    float lse2;          // log-sum-exp of the row times log2(e)
+    int token;           // in [0, V)
+    float g_token;       // g (1 - p_token), formed in fp64: the target's own gradient entry
+};
+
+// ------------------------------------------------------------------------------------------------------
+// Step 2: one warp per row.  Rows beyond T (padding of the last 128-row block) get a zero record.
+// ------------------------------------------------------------------------------------------------------
+struct TermsArgs {
+    const uint16_t* hidden;
+    int64_t ldh;
+    const uint16_t* W;
+    int64_t ldw;
+    const float2* partial;
+    int32_t n_parts;
+    int64_t rows_padded;
+    pods_loss::RowArgs row;      // tokens, old/ref log-probs, advantages, weights, mask, T, V, eps, beta, grad_scale, logp
+    int32_t d;
+    RowGrad* grad;               // [rows_padded]
+};
+
+__global__ void __launch_bounds__(256)
+lm_head_row_terms_kernel(const TermsArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= a.rows_padded) return;
+    if (t >= a.row.T) {
+        if (lane == 0) a.grad[t] = RowGrad{0.0f, 0.0f, 0, 0.0f};
+        return;
+    }
+    int tok = a.row.tokens[t];
+    if (tok < 0 || tok >= a.row.V) { tok = 0; if (lane == 0) pods_raise(a.row.status, PODS_STATUS_TOKEN_RANGE); }
+    double lse;
+    float x_tok;
+    merge_row(a.hidden, a.ldh, a.W, a.ldw, t, tok, a.d, a.partial, a.n_parts, a.rows_padded, lane, &lse, &x_tok);
+    if (lane == 0) {
+        const double logp = (double)x_tok - lse;
+        const pods_loss::RowInputs in = pods_loss::load_row_inputs(a.row, t);
+        const pods_loss::TokenTerms tt = pods_loss::token_terms(logp, in, a.row.eps, a.row.beta, a.row.grad_scale);
+        a.row.logp[t] = (float)logp;
+        a.row.row_loss[t] = tt.weighted_loss;
+        RowGrad r;
+        r.g = (float)tt.g;
+        r.lse2 = (float)(lse * 1.4426950408889634);
+        r.token = tok;
+        r.g_token = (float)(tt.g * -expm1(logp));
+        a.grad[t] = r;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Step 3: the panel's logits again, turned into the gradient with respect to the logits on the way out.
+// ------------------------------------------------------------------------------------------------------
+struct DlogitsArgs {
+    int32_t V, d;
+    int32_t n_row_blocks;
+    int32_t tile0;               // first 256-column tile of the panel, counted over the whole vocabulary
+    int32_t n_col_tiles;         // tiles of this panel
+    int32_t tiles_per_part;
+    int64_t n_items;             // parts x row blocks, part-major
+    const RowGrad* grad;         // [n_row_blocks * 128]
+    uint16_t* panel;             // bf16 [n_row_blocks * 128, ldp]
+    int64_t ldp;                 // >= n_col_tiles * 256
+    uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                       const DlogitsArgs a) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* const tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers& bar = *reinterpret_cast<Barriers*>(tiles + (size_t)kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_blocks = (a.d + BK - 1) / BK;
+    const uint32_t tmem_base = pipeline_setup(bar, warp);
+    bool timed_out = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int64_t loads = 0;
+            for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+                const int part = (int)(item / a.n_row_blocks), rb = (int)(item % a.n_row_blocks);
+                const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
+                for (int ct = t0; ct < t1; ++ct) {
+                    for (int kb = 0; kb < k_blocks; ++kb) {
+                        if (!mbar_wait(&bar.empty[stage], phase ^ 1u, timed_out)) timed_out = true;
+                        unsigned char* sa = tiles + (size_t)stage * kStageBytes;
+                        mbar_expect_tx(&bar.full[stage], kStageBytes);
+                        tma_load_tile(sa, &map_hidden, kb * BK, rb * BM, &bar.full[stage]);
+                        tma_load_tile(sa + kStageBytesA, &map_w, kb * BK, (a.tile0 + ct) * BN, &bar.full[stage]);
+                        ++loads;
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!drain_loads(bar, loads)) timed_out = true;
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+                const int part = (int)(item / a.n_row_blocks);
+                const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
+                for (int ct = t0; ct < t1; ++ct) {
+                    if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
+                    tcgen05_fence_after();
+                    const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
+                    for (int kb = 0; kb < k_blocks; ++kb) {
+                        if (!mbar_wait(&bar.full[stage], phase, timed_out)) timed_out = true;
+                        tcgen05_fence_after();
+                        const uint32_t sa = smem_u32(tiles + (size_t)stage * kStageBytes);
+                        const uint64_t da = smem_desc_k_major(sa), db = smem_desc_k_major(sa + kStageBytesA);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            umma(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 >> 4), db + (uint64_t)(k * UMMA_K * 2 >> 4),
+                                 instr_desc(false, false), (kb | k) != 0 ? 1u : 0u);
+                        umma_commit(&bar.empty[stage]);
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    umma_commit(&bar.acc_full[acc]);
+                    if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // epilogue: thread r of the four warps owns row r of the tile
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+            const int part = (int)(item / a.n_row_blocks), rb = (int)(item % a.n_row_blocks);
+            const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
+            const int64_t row = (int64_t)rb * BM + row_in_tile;
+            const RowGrad rg = a.grad[PODS_CLAMPED(row, (int64_t)a.n_row_blocks * BM, a.status)];
+            const float neg_g = -rg.g;
+            uint16_t* const out_row = a.panel + row * a.ldp;
+            for (int ct = t0; ct < t1; ++ct) {
+                if (!mbar_wait(&bar.acc_full[acc], acc_phase, timed_out)) timed_out = true;
+                tcgen05_fence_after();
+                const int col0 = (a.tile0 + ct) * BN;                     // vocabulary entry of the tile's first column
+                const int valid_cols = min(BN, a.V - col0);              // beyond the vocabulary the gradient is 0
+                const int tok_col = rg.token - col0;                     // the target's column in this tile, if inside
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    float v[32];
+                    tmem_load_32(tmem_base + lane_addr + (uint32_t)(acc * BN + c0), v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = neg_g * ex2(fmaf(v[i], kLog2e, -rg.lse2));
+                    if (c0 + 32 > valid_cols) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = (c0 + i < valid_cols) ? v[i] : 0.0f;
+                    }
+                    if ((unsigned)(tok_col - c0) < 32u) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = (tok_col - c0 == i) ? rg.g_token : v[i];
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(out_row + (int64_t)ct * BN + c0);
+                    if (PODS_INDEX_OK((int64_t)ct * BN + c0 + 31, a.ldp, a.status)) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            dst[q] = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                                                pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+                    }
+                }
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.acc_empty[acc]);
+                if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    }
+    if (timed_out && lane == 0) pods_raise(a.status, PODS_STATUS_TIMEOUT);
+    pipeline_teardown(tmem_base, warp);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Steps 4 and 5: C[m, n] (+)= sum_k A[m, k] B[k, n] with C fp32 row-major, B stored by rows of n (MN-major) and
+// A stored either by rows of k (A_MN = false: the panel as it is) or by rows of m (A_MN = true: the panel
+// transposed, read in place).
+// ------------------------------------------------------------------------------------------------------
+struct GemmArgs {
+    int32_t m_tiles, n_tiles, k_blocks;
+    int32_t b_k0;                // first contraction row of B inside its matrix
+    int64_t m_valid, n_valid;    // rows and columns of C that exist
+    float* C;
+    int64_t ldc;
+    int32_t accumulate;          // 0: C = product, 1: C += product
+    uint32_t* status;
+};
+
+template <bool A_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                         const GemmArgs g) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* const tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers& bar = *reinterpret_cast<Barriers*>(tiles + (size_t)kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tmem_base = pipeline_setup(bar, warp);
+    const int64_t n_tiles_total = (int64_t)g.m_tiles * g.n_tiles;
+    bool timed_out = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int64_t loads = 0;
+            for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+                const int m0 = (int)(tile / g.n_tiles) * BM, n0 = (int)(tile % g.n_tiles) * BN;
+                for (int kb = 0; kb < g.k_blocks; ++kb) {
+                    if (!mbar_wait(&bar.empty[stage], phase ^ 1u, timed_out)) timed_out = true;
+                    unsigned char* sa = tiles + (size_t)stage * kStageBytes;
+                    mbar_expect_tx(&bar.full[stage], kStageBytes);
+                    if (A_MN) {
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i)
+                            tma_load_tile(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage]);
+                    } else {
+                        tma_load_tile(sa, &map_a, kb * BK, m0, &bar.full[stage]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < BN / 64; ++i)
+                        tma_load_tile(sa + kStageBytesA + i * kBoxBytes, &map_b, n0 + 64 * i, g.b_k0 + kb * BK, &bar.full[stage]);
+                    ++loads;
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!drain_loads(bar, loads)) timed_out = true;
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            constexpr uint32_t idesc = instr_desc(A_MN, true);
+            // 16 contraction entries further: 32 bytes along a K-major row, 16 rows of 128 bytes in an MN-major box
+            constexpr uint64_t a_step = A_MN ? (uint64_t)(UMMA_K * 128 >> 4) : (uint64_t)(UMMA_K * 2 >> 4);
+            constexpr uint64_t b_step = (uint64_t)(UMMA_K * 128 >> 4);
+            for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+                if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
+                tcgen05_fence_after();
+                const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < g.k_blocks; ++kb) {
+                    if (!mbar_wait(&bar.full[stage], phase, timed_out)) timed_out = true;
+                    tcgen05_fence_after();
+                    const uint32_t sa = smem_u32(tiles + (size_t)stage * kStageBytes);
+                    const uint64_t da = A_MN ? smem_desc_mn_major(sa) : smem_desc_k_major(sa);
+                    const uint64_t db = smem_desc_mn_major(sa + kStageBytesA);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma(tmem_acc, da + a_step * k, db + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(&bar.empty[stage]);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                umma_commit(&bar.acc_full[acc]);
+                if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+            const int64_t row = (int64_t)(tile / g.n_tiles) * BM + row_in_tile;
+            const int n0 = (int)(tile % g.n_tiles) * BN;
+            const bool row_ok = row < g.m_valid;
+            float* const c_row = g.C + (row_ok ? row : 0) * g.ldc;
+            if (!mbar_wait(&bar.acc_full[acc], acc_phase, timed_out)) timed_out = true;
+            tcgen05_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                float v[32];
+                tmem_load_32(tmem_base + lane_addr + (uint32_t)(acc * BN + c0), v);
+                if (row_ok) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int col = n0 + c0 + 4 * q;
+                        if (col + 3 < g.n_valid) {
+                            float4* p = reinterpret_cast<float4*>(c_row + col);
+                            float4 o = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                            if (g.accumulate) {
+                                const float4 old = *p;
+                                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                            }
+                            *p = o;
+                        }
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar.acc_empty[acc]);
+            if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+    if (timed_out && lane == 0) pods_raise(g.status, PODS_STATUS_TIMEOUT);
+    pipeline_teardown(tmem_base, warp);
+}
+
+// How a call is cut up: the statistics plan, the panels of the vocabulary and the workspace regions.
+struct Layout {
+    Plan stats;                  // statistics pass over the whole vocabulary
+    int64_t rows_padded;         // T rounded up to whole 128-row blocks
+    int total_tiles;             // 256-column tiles of the vocabulary
+    int tiles_per_panel, n_panels;
+    int64_t ldp;                 // panel row pitch in elements = tiles_per_panel * 256
+    size_t off_row_loss, off_grad, off_panel, bytes;
+};
+
+Layout make_layout(int64_t T, int32_t V, int sms) {
+    Layout l;
+    l.stats = make_plan(T, V, sms);
+    l.rows_padded = (int64_t)l.stats.n_row_blocks * BM;
+    l.total_tiles = l.stats.n_col_tiles;
+    int64_t max_tiles = (int64_t)(g_panel_bytes / ((size_t)l.rows_padded * BN * 2));
+    if (max_tiles < 1) max_tiles = 1;
+    l.n_panels = (int)((l.total_tiles + max_tiles - 1) / max_tiles);
+    l.tiles_per_panel = (l.total_tiles + l.n_panels - 1) / l.n_panels;
+    l.ldp = (int64_t)l.tiles_per_panel * BN;
+    size_t off = align_up((size_t)l.stats.n_parts * (size_t)l.rows_padded * sizeof(float2), 256);
+    l.off_row_loss = off;
+    off += align_up((size_t)T * sizeof(double), 256);
+    l.off_grad = off;
+    off += align_up((size_t)l.rows_padded * sizeof(RowGrad), 256);
+    l.off_panel = off;
+    off += align_up((size_t)l.rows_padded * (size_t)l.ldp * 2, 256);
+    l.bytes = off;
+    return l;
+}
+
+template <bool A_MN>
+int launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmArgs& g, int sms, cudaStream_t s) {
+    const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
+    if (tiles <= 0 || g.k_blocks <= 0) return PODS_OK;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_grad_gemm_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    lm_head_grad_gemm_kernel<A_MN><<<(int)(tiles < sms ? tiles : sms), kThreads, kSmemBytes, s>>>(map_a, map_b, g);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    return PODS_OK;
+}
+
+}  // namespace
+
+extern "C" size_t pods_set_loss_from_hidden_panel_bytes(size_t bytes) {
+    const size_t before = g_panel_bytes;
+    g_panel_bytes = bytes < (size_t)65536 ? (size_t)65536 : bytes;
+    return before;
+}
+
+extern "C" size_t grpo_loss_from_hidden_workspace_bytes(int64_t T, int32_t V, int32_t d) {
+    (void)d;
+    if (T <= 0 || V <= 0) return 0;
+    return make_layout(T, V, pods_sm_count()).bytes;
+}
+
+extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_t ldw, const int32_t* tokens,
+                                     const float* old_logp, const float* ref_logp, const float* adv,
+                                     const double* seq_weight, const int64_t* cu_seqlens, int64_t M, int64_t row0,
+                                     const uint8_t* mask, int64_t T, int32_t V, int32_t d, float eps, float beta,
+                                     float grad_scale, double* loss_acc, float* logp, float* dhidden, int64_t lddh,
+                                     float* dW, int64_t lddw, void* workspace, size_t workspace_bytes,
+                                     uint32_t* status, void* stream) {
+    if (T < 0 || V < 1 || M < 1 || row0 < 0 || d < 8 || d % 8 != 0 || ldh < d || ldw < d || ldh % 8 != 0 ||
+        ldw % 8 != 0 || lddh < d || lddw < d || lddh % 4 != 0 || lddw % 4 != 0)
+        return PODS_ERR_INVALID_ARG;
+    if (!(eps >= 0.0f) || !(beta == beta)) return PODS_ERR_INVALID_ARG;
+    if (T == 0) return PODS_OK;
+    if (hidden == nullptr || W == nullptr || tokens == nullptr || old_logp == nullptr || adv == nullptr ||
+        seq_weight == nullptr || cu_seqlens == nullptr || loss_acc == nullptr || logp == nullptr ||
+        dhidden == nullptr || dW == nullptr)
+        return PODS_ERR_INVALID_ARG;
+    if (ref_logp == nullptr && beta != 0.0f) return PODS_ERR_INVALID_ARG;
+    if (!pods_aligned(hidden, 16) || !pods_aligned(W, 16) || !pods_aligned(dhidden, 16) || !pods_aligned(dW, 16) ||
+        !pods_aligned(loss_acc, 8) || !pods_aligned(logp, 4))
+        return PODS_ERR_INVALID_ARG;
+    const int sms = pods_sm_count();
+    const Layout l = make_layout(T, V, sms);
+    if (workspace == nullptr || workspace_bytes < l.bytes || !pods_aligned(workspace, 256)) return PODS_ERR_WORKSPACE;
+
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    float2* partial = reinterpret_cast<float2*>(ws);
+    double* row_loss = reinterpret_cast<double*>(ws + l.off_row_loss);
+    RowGrad* grad = reinterpret_cast<RowGrad*>(ws + l.off_grad);
+    uint16_t* panel = reinterpret_cast<uint16_t*>(ws + l.off_panel);
+    cudaStream_t s = pods_stream(stream);
+
+    // 1. statistics of every row over the whole vocabulary
+    int rc = launch_lm_head_stats(hidden, ldh, W, ldw, T, V, d, l.stats, partial, status, s);
+    if (rc != PODS_OK) return rc;
+
+    // 2. log-probs, loss terms, gradient factors
+    TermsArgs ta;
+    ta.hidden = static_cast<const uint16_t*>(hidden);
+    ta.ldh = ldh;
+    ta.W = static_cast<const uint16_t*>(W);
+    ta.ldw = ldw;
+    ta.partial = partial;
+    ta.n_parts = l.stats.n_parts;
+    ta.rows_padded = l.rows_padded;
+    ta.d = d;
+    ta.grad = grad;
+    pods_loss::RowArgs& a = ta.row;
+    a.logits = nullptr;
+    a.ldl = 0;
+    a.tokens = tokens;
+    a.old_logp = old_logp;
+    a.ref_logp = ref_logp;
+    a.adv = adv;
+    a.seq_weight = seq_weight;
+    a.cu_seqlens = cu_seqlens;
+    a.M = M;
+    a.row0 = row0;
+    a.mask = mask;
+    a.T = T;
+    a.V = V;
+    a.eps = eps;
+    a.beta = beta;
+    a.grad_scale = grad_scale;
+    a.logp = logp;
+    a.dlogits = nullptr;
+    a.ldd = 0;
+    a.row_loss = row_loss;
+    a.prep = nullptr;
+    a.status = status;
+    a.vec_ok = 0;
+    a.precise = 0;
+    const int warps_per_block = 8;
+    lm_head_row_terms_kernel<<<(unsigned)((l.rows_padded + warps_per_block - 1) / warps_per_block), warps_per_block * 32, 0, s>>>(ta);
+    PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+    rc = pods_loss::launch_loss_reduce(row_loss, T, loss_acc, s);
+    if (rc != PODS_OK) return rc;
+
+    // 3-5. panel by panel
+    CUtensorMap map_h_rows, map_w_rows;          // hidden / W tiles by rows of d: K-major operands of the logits
+    CUtensorMap map_w_box, map_h_box;            // the same matrices in 64 x 64 boxes: MN-major B operands
+    CUtensorMap map_panel_rows, map_panel_box;   // the panel as K-major A (dhidden) and as MN-major A (dW)
+    if ((rc = make_map(&map_h_rows, hidden, T, d, ldh, BM)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_w_rows, W, V, d, ldw, BN)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_w_box, W, V, d, ldw, 64)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_h_box, hidden, T, d, ldh, 64)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_panel_rows, panel, l.rows_padded, l.ldp, l.ldp, BM)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_panel_box, panel, l.rows_padded, l.ldp, l.ldp, 64)) != PODS_OK) return rc;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_dlogits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+
+    for (int p = 0; p < l.n_panels; ++p) {
+        const int tile0 = p * l.tiles_per_panel;
+        const int n_tiles = (l.total_tiles - tile0 < l.tiles_per_panel) ? l.total_tiles - tile0 : l.tiles_per_panel;
+        if (n_tiles <= 0) break;
+        const int64_t cols = (int64_t)n_tiles * BN;
+        const Plan pp = make_plan(T, cols, sms);
+
+        DlogitsArgs da;
+        da.V = V;
+        da.d = d;
+        da.n_row_blocks = pp.n_row_blocks;
+        da.tile0 = tile0;
+        da.n_col_tiles = n_tiles;
+        da.tiles_per_part = pp.tiles_per_part;
+        da.n_items = (int64_t)pp.n_parts * pp.n_row_blocks;
+        da.grad = grad;
+        da.panel = panel;
+        da.ldp = l.ldp;
+        da.status = status;
+        lm_head_dlogits_kernel<<<pp.grid, kThreads, kSmemBytes, s>>>(map_h_rows, map_w_rows, da);
+        PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
+
+        GemmArgs gh;                             // dhidden[T, d] (+)= panel[T, cols] . W[tile0 * 256 + (0 .. cols), d]
+        gh.m_tiles = pp.n_row_blocks;
+        gh.n_tiles = (d + BN - 1) / BN;
+        gh.k_blocks = (int)(cols / BK);
+        gh.b_k0 = tile0 * BN;
+        gh.m_valid = T;
+        gh.n_valid = d;
+        gh.C = dhidden;
+        gh.ldc = lddh;
+        gh.accumulate = p > 0 ? 1 : 0;
+        gh.status = status;
+        if ((rc = launch_gemm<false>(map_panel_rows, map_w_box, gh, sms, s)) != PODS_OK) return rc;
+
+        GemmArgs gw;                             // dW[tile0 * 256 + (0 .. cols), d] += panel^T . hidden
+        gw.m_tiles = (int)(cols / BM);
+        gw.n_tiles = (d + BN - 1) / BN;
+        gw.k_blocks = (int)(l.rows_padded / BK);
+        gw.b_k0 = 0;
+        gw.m_valid = (int64_t)V - (int64_t)tile0 * BN < cols ? (int64_t)V - (int64_t)tile0 * BN : cols;
+        gw.n_valid = d;
+        gw.C = dW + (int64_t)tile0 * BN * lddw;
+        gw.ldc = lddw;
+        gw.accumulate = 1;
+        gw.status = status;
+        if ((rc = launch_gemm<true>(map_panel_box, map_h_box, gw, sms, s)) != PODS_OK) return rc;
+    }
+    return PODS_OK;
+}

@@ -1,0 +1,203 @@
+"""grpo_loss_from_hidden (CUDA, tensor cores) against the fp64 oracle: the objective on logits = hidden W^T and its
+gradient with respect to hidden and W, the [T,V] logits and their gradient never stored in full.
+
+Tolerances.  logp abs <= 1e-3 and the loss as everywhere else.  The gradients are sums of products
+dlogits[t,v] W[v,j] (over v) and dlogits[t,v] hidden[t,j] (over t) in which the kernel rounds dlogits to bf16 - as the
+unfused path's stored gradient is - so every term carries a relative error of at most 2^-9; the fp32 evaluation of the
+softmax (logits accumulated in fp32 over d terms, the fp32 log-sum-exp) and the fp32 accumulation of the sums add a
+few 1e-5 relative to the terms.  Hence, element by element,
+    |gpu - oracle| <= 2^-8 * sum |dlogits| |W|      (dhidden)        2^-8 * sum |dlogits| |hidden|      (dW),
+the sums of magnitudes coming from the oracle.  The bound assumes that no row's factor g_t is itself a cancellation
+(reading of the dlogits tolerance for the unfused kernel); the inputs are drawn so that there is none, which is asserted.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import lm_head
+from paper_2504_13818_b200 import binding
+from parity import LOGP_ATOL, LOSS_RTOL, record
+
+pytestmark = pytest.mark.gpu
+
+GRAD_RTOL = 2.0 ** -8
+EPS, BETA = 0.2, 0.04
+
+
+def _inputs(T, V, d, M, seed, masked=(), zero_adv=()):
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    hidden = torch.randn((T, d), generator=gen, device=dev).to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=gen, device=dev) * (3.0 / d ** 0.5)).to(torch.bfloat16)
+    tokens = torch.randint(0, V, (T,), generator=gen, device=dev, dtype=torch.int32)
+    rng = np.random.default_rng(seed)
+    cuts = np.sort(rng.choice(np.arange(1, T), size=min(M - 1, T - 1), replace=False)) if M > 1 else np.array([], int)
+    cu = np.concatenate([[0], cuts, [T]]).astype(np.int64)
+    M = cu.shape[0] - 1
+    adv = rng.normal(size=M)
+    adv = (np.sign(adv) * (0.2 + np.abs(adv))).astype(np.float32)  # away from 0: a tiny advantage could cancel the KL term
+    adv[list(zero_adv)] = 0.0
+    mask = np.ones(T, np.uint8)
+    mask[list(masked)] = 0
+    hb = hidden.view(torch.uint16).cpu().numpy()
+    wb = W.view(torch.uint16).cpu().numpy()
+    tok = tokens.cpu().numpy()
+    base = lm_head.logp_from_hidden(hb, wb, tok)["logp"]
+    old = (base + rng.normal(0, 0.15, T)).astype(np.float32)
+    # the reference log-prob stays at least 0.02 away from the policy's: no row factor is a cancellation
+    noise = rng.normal(0, 0.1, T)
+    ref = (base + np.sign(noise) * (0.02 + np.abs(noise))).astype(np.float32)
+    return dict(hidden=hidden, W=W, tokens=tokens, hb=hb, wb=wb, tok=tok, cu=cu, adv=adv, mask=mask, old=old, ref=ref,
+                T=T, V=V, d=d, M=M)
+
+
+def _oracle(c, beta=BETA):
+    sw = oracle.seq_weights(c["mask"], c["cu"])
+    out = lm_head.loss_grad_from_hidden(c["hb"], c["wb"], c["tok"], c["old"], c["ref"] if beta != 0 else None, c["adv"],
+                                        sw, oracle.seq_of_rows(c["cu"]), c["mask"], EPS, beta)
+    out["loss"] = oracle.grpo_loss(out["ell"], c["mask"], c["cu"])
+    return out
+
+
+def _run(c, beta=BETA, dW=None, grad_scale=1.0, hidden=None, W=None):
+    dev = c["hidden"].device
+    cu = torch.from_numpy(c["cu"]).to(dev)
+    mask = torch.from_numpy(c["mask"]).to(dev)
+    sw = torch.empty(c["M"], dtype=torch.float64, device=dev)
+    binding.grpo_seq_weights(mask, cu, sw)
+    loss_acc = torch.zeros(1, dtype=torch.float64, device=dev)
+    if dW is None:
+        dW = torch.zeros((c["V"], c["d"]), dtype=torch.float32, device=dev)
+    status = binding.new_status()
+    logp, dh = binding.grpo_loss_from_hidden(
+        c["hidden"] if hidden is None else hidden, c["W"] if W is None else W, c["tokens"],
+        torch.from_numpy(c["old"]).to(dev), torch.from_numpy(c["ref"]).to(dev) if beta != 0 else None,
+        torch.from_numpy(c["adv"]).to(dev), sw, cu, 0, mask, EPS, beta, loss_acc, dW, grad_scale=grad_scale, status=status)
+    torch.cuda.synchronize()
+    return dict(logp=logp.cpu().numpy(), dhidden=dh.cpu().numpy().astype(np.float64),
+                dW=dW.cpu().numpy().astype(np.float64), loss=float(loss_acc.item()), status=binding.read_status(status))
+
+
+def _no_cancelling_factor(c, want):
+    """|dg/dlogp| * 2e-6 / |g| stays far below the bf16 grain on every live row with a gradient."""
+    sw = oracle.seq_weights(c["mask"], c["cu"])[oracle.seq_of_rows(c["cu"])] * (c["mask"] != 0)
+    a = c["adv"][oracle.seq_of_rows(c["cu"])].astype(np.float64)
+    rho = np.exp(want["logp"] - c["old"].astype(np.float64))
+    ed = np.exp(c["ref"].astype(np.float64) - want["logp"])
+    flows = rho * a <= np.clip(rho, 1 - float(np.float32(EPS)), 1 + float(np.float32(EPS))) * a   # not on the clipped side
+    dg = 2e-6 * sw * (np.abs(a) * rho * flows + BETA * ed)
+    g = np.abs(want["g"])
+    rel = np.where(g > 0, dg / np.where(g > 0, g, 1.0), 0.0)
+    return float(rel.max())
+
+
+def _compare(case, got, want, c, scale=1.0):
+    assert got["status"] == 0
+    logp_err = float(np.abs(got["logp"] - want["logp"]).max())
+    dh_ratio = float((np.abs(got["dhidden"] - scale * want["dhidden"]) / (scale * want["abs_dhidden"] + 1e-30)).max())
+    dw_ratio = float((np.abs(got["dW"] - scale * want["dW"]) / (scale * want["abs_dW"] + 1e-30)).max())
+    loss_rel = abs(got["loss"] - want["loss"]) / max(abs(want["loss"]), 1e-300)
+    record(case, logp_abs=logp_err, dhidden_over_term_sum=dh_ratio, dW_over_term_sum=dw_ratio, loss_rel_literal=loss_rel,
+           bound=GRAD_RTOL)
+    assert logp_err <= LOGP_ATOL
+    assert dh_ratio <= GRAD_RTOL, "dhidden off by %.3g of its term sum" % dh_ratio
+    assert dw_ratio <= GRAD_RTOL, "dW off by %.3g of its term sum" % dw_ratio
+    # where nothing is contracted the gradient is exactly zero: masked rows, vocabulary rows no live row reaches
+    dead = want["abs_dhidden"].max(axis=1) == 0
+    assert (got["dhidden"][dead] == 0).all()
+    return loss_rel
+
+
+@pytest.mark.parametrize("T,V,d,M", [(64, 1024, 128, 3),       # one block of rows, four tiles, one panel
+                                     (128, 256, 64, 1),        # exactly one tile, one k-block
+                                     (300, 1000, 72, 5),       # ragged rows, vocabulary and features
+                                     (1, 8, 8, 1),             # the smallest legal shape
+                                     (515, 5000, 320, 7),      # several row blocks; d beyond one 256-column tile
+                                     (512, 32000, 1024, 16)])
+def test_loss_and_gradients_against_the_oracle(T, V, d, M):
+    masked = (0, T // 2) if T > 4 else ()
+    c = _inputs(T, V, d, M, seed=T + V + d, masked=masked, zero_adv=(0,) if M > 2 else ())
+    want = _oracle(c)
+    assert _no_cancelling_factor(c, want) < 2.0 ** -11
+    got = _run(c)
+    loss_rel = _compare("grpo_loss_from_hidden T=%d V=%d d=%d" % (T, V, d), got, want, c)
+    scale = np.abs(want["ell"]).mean()
+    assert abs(got["loss"] - want["loss"]) <= LOSS_RTOL * max(abs(want["loss"]), scale / 1e3), loss_rel
+
+
+def test_several_panels_accumulate_to_the_same_result():
+    """With the panel limit at its minimum every 256-column tile is a panel of its own: dhidden is accumulated over
+    all of them, dW is assembled from them."""
+    c = _inputs(300, 1500, 96, 4, seed=21)
+    want = _oracle(c)
+    one = _run(c)
+    before = binding.set_loss_from_hidden_panel_bytes(1)
+    try:
+        many = _run(c)
+    finally:
+        binding.set_loss_from_hidden_panel_bytes(before)
+    _compare("grpo_loss_from_hidden six panels", many, want, c)
+    assert one["logp"].tobytes() == many["logp"].tobytes() and one["loss"] == many["loss"]
+    assert one["dW"].tobytes() == many["dW"].tobytes()              # a tile's dW does not depend on the panelling
+    assert np.abs(one["dhidden"] - many["dhidden"]).max() <= 1e-5 * np.abs(want["abs_dhidden"]).max()
+
+
+def test_dw_accumulates_and_grad_scale_scales():
+    c = _inputs(200, 777 * 8, 64, 3, seed=22)
+    want = _oracle(c)
+    dev = c["hidden"].device
+    dW = torch.zeros((c["V"], c["d"]), dtype=torch.float32, device=dev)
+    first = _run(c, dW=dW)
+    second = _run(c, dW=dW, grad_scale=0.5)                          # the same buffer again: 1 + 0.5 times the gradient
+    np.testing.assert_allclose(second["dW"], 1.5 * first["dW"], rtol=0, atol=2e-6 * np.abs(first["dW"]).max())
+    half = _run(c, grad_scale=0.5)
+    _compare("grpo_loss_from_hidden grad_scale 0.5", half, want, c, scale=0.5)
+    assert half["loss"] == first["loss"]
+
+
+def test_without_kl_strided_inputs_and_token_range():
+    c = _inputs(130, 520, 96, 2, seed=23)
+    dev = c["hidden"].device
+    wide_h = torch.zeros((c["T"], c["d"] + 8), dtype=torch.bfloat16, device=dev)
+    wide_w = torch.zeros((c["V"], c["d"] + 16), dtype=torch.bfloat16, device=dev)
+    wide_h[:, :c["d"]] = c["hidden"]
+    wide_w[:, :c["d"]] = c["W"]
+    want = _oracle(c, beta=0.0)
+    got = _run(c, beta=0.0, hidden=wide_h[:, :c["d"]], W=wide_w[:, :c["d"]])
+    _compare("grpo_loss_from_hidden beta=0, pitched rows", got, want, c)
+    tok = c["tokens"].clone()
+    tok[3] = c["V"]
+    c2 = dict(c, tokens=tok)
+    bad = _run(c2, beta=0.0)
+    assert bad["status"] == binding.STATUS_TOKEN_RANGE
+    tok0 = c["tok"].copy()
+    tok0[3] = 0
+    want0 = _oracle(dict(c, tok=tok0), beta=0.0)
+    assert np.abs(bad["logp"] - want0["logp"]).max() <= LOGP_ATOL
+
+
+def test_repeated_calls_give_the_same_bits():
+    c = _inputs(384, 5000, 192, 5, seed=24)
+    a, b = _run(c), _run(c)
+    for k in ("logp", "dhidden", "dW"):
+        assert a[k].tobytes() == b[k].tobytes()
+    assert a["loss"] == b["loss"]
+
+
+@pytest.mark.skipif(not torch.cuda.is_available() or torch.cuda.get_device_properties(0).total_memory < 20e9,
+                    reason="needs a few GB of device memory")
+def test_qwen_vocabulary_at_d_2048():
+    """The vocabulary and width of the 3B policy on 512 rows (the oracle's five fp64 products take about a minute),
+    with the panel limit lowered so that the vocabulary is cut into several panels as it is at 16384 rows."""
+    c = _inputs(512, 151936, 2048, 8, seed=25)
+    want = _oracle(c)
+    assert _no_cancelling_factor(c, want) < 2.0 ** -11
+    before = binding.set_loss_from_hidden_panel_bytes(40 << 20)
+    try:
+        got = _run(c)
+    finally:
+        binding.set_loss_from_hidden_panel_bytes(before)
+    _compare("grpo_loss_from_hidden T=512 V=151936 d=2048", got, want, c)
+    assert abs(got["loss"] - want["loss"]) <= LOSS_RTOL * max(abs(want["loss"]), np.abs(want["ell"]).mean() / 1e3)
