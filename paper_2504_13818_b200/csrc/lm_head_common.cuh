@@ -70,6 +70,20 @@ __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map,
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
+// The same with an L2 eviction policy for the lines the load brings in.
+__device__ __forceinline__ void tma_load_tile_hint(void* dst, const CUtensorMap* map, int x, int y, void* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+// L2 policy for data that streams through once: first in line for eviction, so that it does not push out the
+// matrices every CTA keeps re-reading.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 // Shared-memory operand descriptors of tcgen05.mma for bf16 blocks stored as rows of 128 bytes with the
 // 128-byte swizzle (what the TMA loads above write).  Common fields: start address / 16 in bits 0-13,
 // descriptor version 1 (bit 46), swizzle mode 2 = 128 bytes (bits 61-63).
@@ -143,10 +157,11 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // Barriers initialised, tensor memory allocated by warp 1 (which also frees it), everything visible to the CTA.
-__device__ __forceinline__ uint32_t pipeline_setup(Barriers& bar, int warp) {
+// `epilogue_warps` warps arrive (one lane each) when an accumulator has been read.
+__device__ __forceinline__ uint32_t pipeline_setup(Barriers& bar, int warp, uint32_t epilogue_warps = 4) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&bar.full[s], 1); mbar_init(&bar.empty[s], 1); }
-        for (int b = 0; b < kAccumulators; ++b) { mbar_init(&bar.acc_full[b], 1); mbar_init(&bar.acc_empty[b], 4); }
+        for (int b = 0; b < kAccumulators; ++b) { mbar_init(&bar.acc_full[b], 1); mbar_init(&bar.acc_empty[b], epilogue_warps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc_all(&bar.tmem_base);

@@ -17,7 +17,7 @@
 //      no transposed copy of anything is made.
 // Roles, barriers and bounded waits are those of the statistics kernel: a TMA producer warp, one thread issuing
 // the MMAs into one of two 256-column accumulators in tensor memory, four epilogue warps (one tile row per
-// thread).  All loads are plain (never multicast) TMA loads of this GPU's own memory.
+// thread; eight warps, half a row per thread, where the epilogue forms the gradient).  All loads are plain (never multicast) TMA loads of this GPU's own memory.
 
 #include "grpo_loss_common.cuh"
 #include "lm_head_common.cuh"
@@ -90,13 +90,27 @@ struct DlogitsArgs {
     int32_t n_row_blocks;
     int32_t tile0;               // first 256-column tile of the panel, counted over the whole vocabulary
     int32_t n_col_tiles;         // tiles of this panel
-    int32_t tiles_per_part;
-    int64_t n_items;             // parts x row blocks, part-major
+    int32_t group_rows;          // row blocks per group of the tile order (see tile_of)
+    int64_t n_items;             // tiles of the panel: column tiles x row blocks
     const RowGrad* grad;         // [n_row_blocks * 128]
-    uint16_t* panel;             // bf16 [n_row_blocks * 128, ldp]
-    int64_t ldp;                 // >= n_col_tiles * 256
+    int64_t ldp;                 // row pitch of the panel (bf16 [n_row_blocks * 128, ldp]), >= n_col_tiles * 256
     uint32_t* status;
 };
+
+// Order of the panel's tiles: groups of `group_rows` blocks of rows; inside a group one column tile after the other,
+// and for each the group's row blocks.  The CTAs that run at the same time (consecutive items) then share a few
+// column tiles of W and a few row blocks of hidden - 17 MB at 16 row blocks per group - instead of sweeping all of
+// hidden (67 MB at 16384 rows, more than one L2 partition holds) for every column tile.
+__device__ __forceinline__ void tile_of(const DlogitsArgs& a, int64_t item, int* ct, int* rb) {
+    const int64_t per_group = (int64_t)a.group_rows * a.n_col_tiles;
+    const int n_groups = (a.n_row_blocks + a.group_rows - 1) / a.group_rows;
+    int g = (int)(item / per_group);
+    if (g > n_groups - 1) g = n_groups - 1;
+    const int64_t rem = item - (int64_t)g * per_group;
+    const int rows_here = min(a.group_rows, a.n_row_blocks - g * a.group_rows);
+    *ct = (int)(rem / rows_here);
+    *rb = g * a.group_rows + (int)(rem % rows_here);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
@@ -104,15 +118,26 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+// Eight epilogue warps here (two per quarter of the TMEM lanes, each taking half of the tile's columns): with four,
+// a warp alone on its scheduler spent about 15 us per tile on the dependent chain load - exponentials - round - store,
+// more than the 12 us the tensor core needs for the tile.
+constexpr int kDlogitsThreads = 64 + 8 * 32;
+// The gradient leaves through shared memory: a warp stages 32 rows x 64 columns (whole 128-byte lines) and one thread
+// sends them off as one bulk tensor store.  Stored straight from registers (16 bytes per lane and instruction, every
+// lane another line) the same data cost 1.5 ms of 7.7 per 16384 rows.
+constexpr uint32_t kStagingBytesPerWarp = 32 * 128;
+constexpr size_t kDlogitsSmemBytes = 1024 + (size_t)kStages * kStageBytes + 8 * kStagingBytesPerWarp + 256;
+
+__global__ void __launch_bounds__(kDlogitsThreads, 1)
 lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                       const DlogitsArgs a) {
+                       const __grid_constant__ CUtensorMap map_panel, const DlogitsArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* const tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Barriers& bar = *reinterpret_cast<Barriers*>(tiles + (size_t)kStages * kStageBytes);
+    unsigned char* const staging = tiles + (size_t)kStages * kStageBytes;        // 1024-byte aligned, 4 KB per warp
+    Barriers& bar = *reinterpret_cast<Barriers*>(staging + 8 * kStagingBytesPerWarp);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_blocks = (a.d + BK - 1) / BK;
-    const uint32_t tmem_base = pipeline_setup(bar, warp);
+    const uint32_t tmem_base = pipeline_setup(bar, warp, 8);
     bool timed_out = false;
 
     if (warp == 0) {
@@ -121,9 +146,9 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
             uint32_t phase = 0;
             int64_t loads = 0;
             for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
-                const int part = (int)(item / a.n_row_blocks), rb = (int)(item % a.n_row_blocks);
-                const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
-                for (int ct = t0; ct < t1; ++ct) {
+                int ct, rb;
+                tile_of(a, item, &ct, &rb);
+                {
                     for (int kb = 0; kb < k_blocks; ++kb) {
                         if (!mbar_wait(&bar.empty[stage], phase ^ 1u, timed_out)) timed_out = true;
                         unsigned char* sa = tiles + (size_t)stage * kStageBytes;
@@ -145,9 +170,7 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
             int acc = 0;
             uint32_t acc_phase = 0;
             for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
-                const int part = (int)(item / a.n_row_blocks);
-                const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
-                for (int ct = t0; ct < t1; ++ct) {
+                {
                     if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
                     tcgen05_fence_after();
                     const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
@@ -170,45 +193,66 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
         }
         __syncwarp();
     } else {
-        // epilogue: thread r of the four warps owns row r of the tile
+        // epilogue: warps 2-9; a warp reads the TMEM lanes of its quarter (warp % 4) and one half of the columns
         const int quarter = warp & 3;
+        const int col_begin = ((warp - 2) >> 2) * (BN / 2);
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        unsigned char* const stage_warp = staging + (size_t)(warp - 2) * kStagingBytesPerWarp;   // 32 lines of 128 bytes
+        unsigned char* const stage_line = stage_warp + lane * 128;
+        const uint64_t stream_policy = l2_policy_evict_first();      // the panel is written once and read much later
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
-            const int part = (int)(item / a.n_row_blocks), rb = (int)(item % a.n_row_blocks);
-            const int t0 = part * a.tiles_per_part, t1 = min(a.n_col_tiles, t0 + a.tiles_per_part);
+            int ct, rb;
+            tile_of(a, item, &ct, &rb);
             const int64_t row = (int64_t)rb * BM + row_in_tile;
             const RowGrad rg = a.grad[PODS_CLAMPED(row, (int64_t)a.n_row_blocks * BM, a.status)];
             const float neg_g = -rg.g;
-            uint16_t* const out_row = a.panel + row * a.ldp;
-            for (int ct = t0; ct < t1; ++ct) {
+            {
                 if (!mbar_wait(&bar.acc_full[acc], acc_phase, timed_out)) timed_out = true;
                 tcgen05_fence_after();
                 const int col0 = (a.tile0 + ct) * BN;                     // vocabulary entry of the tile's first column
                 const int valid_cols = min(BN, a.V - col0);              // beyond the vocabulary the gradient is 0
                 const int tok_col = rg.token - col0;                     // the target's column in this tile, if inside
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    float v[32];
-                    tmem_load_32(tmem_base + lane_addr + (uint32_t)(acc * BN + c0), v);
+                for (int c0 = col_begin; c0 < col_begin + BN / 2; c0 += 64) {
+                    // 64 columns = one 128-byte line of the panel per row; the warp's 32 lines are staged in shared
+                    // memory (16-byte pieces swizzled as the store's tensor map expects) and leave as one bulk store
+                    uint4 q[8];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = neg_g * ex2(fmaf(v[i], kLog2e, -rg.lse2));
-                    if (c0 + 32 > valid_cols) {
+                    for (int h = 0; h < 2; ++h) {
+                        const int c = c0 + 32 * h;
+                        float v[32];
+                        tmem_load_32(tmem_base + lane_addr + (uint32_t)(acc * BN + c), v);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = (c0 + i < valid_cols) ? v[i] : 0.0f;
+                        for (int i = 0; i < 32; ++i) v[i] = neg_g * ex2(fmaf(v[i], kLog2e, -rg.lse2));
+                        if (c + 32 > valid_cols) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = (c + i < valid_cols) ? v[i] : 0.0f;
+                        }
+                        if ((unsigned)(tok_col - c) < 32u) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = (tok_col - c == i) ? rg.g_token : v[i];
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            q[4 * h + j] = make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                                                      pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
                     }
-                    if ((unsigned)(tok_col - c0) < 32u) {
+                    // the previous store must have finished reading the staging lines before they are overwritten
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = (tok_col - c0 == i) ? rg.g_token : v[i];
-                    }
-                    uint4* dst = reinterpret_cast<uint4*>(out_row + (int64_t)ct * BN + c0);
-                    if (PODS_INDEX_OK((int64_t)ct * BN + c0 + 31, a.ldp, a.status)) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            dst[q] = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
-                                                pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4*>(stage_line + ((j ^ (lane & 7)) << 4)) = q[j];
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0 && PODS_INDEX_OK((int64_t)ct * BN + c0 + 63, a.ldp, a.status)) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
+                                     ::"l"(reinterpret_cast<uint64_t>(&map_panel)), "r"(ct * BN + c0),
+                                       "r"(rb * BM + quarter * 32), "r"(smem_u32(stage_warp)), "l"(stream_policy) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
                 tcgen05_fence_before();
@@ -218,6 +262,8 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
             }
         }
     }
+    // a warp's bulk stores must be complete before its shared memory goes away
+    if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (timed_out && lane == 0) pods_raise(a.status, PODS_STATUS_TIMEOUT);
     pipeline_teardown(tmem_base, warp);
 }
@@ -254,6 +300,7 @@ lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             int stage = 0;
             uint32_t phase = 0;
             int64_t loads = 0;
+            const uint64_t stream_policy = l2_policy_evict_first();  // the panel streams through; W and hidden are re-read
             for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
                 const int m0 = (int)(tile / g.n_tiles) * BM, n0 = (int)(tile % g.n_tiles) * BN;
                 for (int kb = 0; kb < g.k_blocks; ++kb) {
@@ -263,9 +310,9 @@ lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
                     if (A_MN) {
 #pragma unroll
                         for (int i = 0; i < BM / 64; ++i)
-                            tma_load_tile(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage]);
+                            tma_load_tile_hint(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage], stream_policy);
                     } else {
-                        tma_load_tile(sa, &map_a, kb * BK, m0, &bar.full[stage]);
+                        tma_load_tile_hint(sa, &map_a, kb * BK, m0, &bar.full[stage], stream_policy);
                     }
 #pragma unroll
                     for (int i = 0; i < BN / 64; ++i)
@@ -361,15 +408,34 @@ struct Layout {
     size_t off_row_loss, off_grad, off_panel, bytes;
 };
 
-Layout make_layout(int64_t T, int32_t V, int sms) {
+// Time of one panel of c column tiles in units of one 128 x 256 x 64 block of tensor-core work: every kernel runs
+// its tiles in waves over the SMs, so what counts is (waves) x (contraction blocks per tile) for the three of them.
+int64_t panel_cost(int64_t c, int64_t row_blocks, int64_t d, int sms) {
+    const int64_t n_d = (d + BN - 1) / BN;
+    const int64_t dlogits = (c * row_blocks + sms - 1) / sms * ((d + BK - 1) / BK);
+    const int64_t dhidden = (row_blocks * n_d + sms - 1) / sms * (c * BN / BK);
+    const int64_t dw = (2 * c * n_d + sms - 1) / sms * (row_blocks * BM / BK);
+    return dlogits + dhidden + dw + 150;             // + three launches' ramp-up and tail
+}
+
+Layout make_layout(int64_t T, int32_t V, int32_t d, int sms) {
     Layout l;
     l.stats = make_plan(T, V, sms);
     l.rows_padded = (int64_t)l.stats.n_row_blocks * BM;
     l.total_tiles = l.stats.n_col_tiles;
     int64_t max_tiles = (int64_t)(g_panel_bytes / ((size_t)l.rows_padded * BN * 2));
     if (max_tiles < 1) max_tiles = 1;
-    l.n_panels = (int)((l.total_tiles + max_tiles - 1) / max_tiles);
-    l.tiles_per_panel = (l.total_tiles + l.n_panels - 1) / l.n_panels;
+    if (max_tiles > l.total_tiles) max_tiles = l.total_tiles;
+    // tiles per panel: the count within the memory limit with the least wave-quantisation loss over the whole call
+    int64_t best = -1;
+    l.tiles_per_panel = (int)max_tiles;
+    for (int64_t c = max_tiles; c >= 1 && c >= max_tiles / 2; --c) {
+        const int64_t full = l.total_tiles / c, rest = l.total_tiles % c;
+        const int64_t cost = full * panel_cost(c, l.stats.n_row_blocks, d, sms) +
+                             (rest ? panel_cost(rest, l.stats.n_row_blocks, d, sms) : 0);
+        if (best < 0 || cost < best) { best = cost; l.tiles_per_panel = (int)c; }
+    }
+    l.n_panels = (l.total_tiles + l.tiles_per_panel - 1) / l.tiles_per_panel;
     l.ldp = (int64_t)l.tiles_per_panel * BN;
     size_t off = align_up((size_t)l.stats.n_parts * (size_t)l.rows_padded * sizeof(float2), 256);
     l.off_row_loss = off;
@@ -401,9 +467,8 @@ extern "C" size_t pods_set_loss_from_hidden_panel_bytes(size_t bytes) {
 }
 
 extern "C" size_t grpo_loss_from_hidden_workspace_bytes(int64_t T, int32_t V, int32_t d) {
-    (void)d;
-    if (T <= 0 || V <= 0) return 0;
-    return make_layout(T, V, pods_sm_count()).bytes;
+    if (T <= 0 || V <= 0 || d <= 0) return 0;
+    return make_layout(T, V, d, pods_sm_count()).bytes;
 }
 
 extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void* W, int64_t ldw, const int32_t* tokens,
@@ -427,7 +492,7 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
         !pods_aligned(loss_acc, 8) || !pods_aligned(logp, 4))
         return PODS_ERR_INVALID_ARG;
     const int sms = pods_sm_count();
-    const Layout l = make_layout(T, V, sms);
+    const Layout l = make_layout(T, V, d, sms);
     if (workspace == nullptr || workspace_bytes < l.bytes || !pods_aligned(workspace, 256)) return PODS_ERR_WORKSPACE;
 
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -487,13 +552,15 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
     CUtensorMap map_h_rows, map_w_rows;          // hidden / W tiles by rows of d: K-major operands of the logits
     CUtensorMap map_w_box, map_h_box;            // the same matrices in 64 x 64 boxes: MN-major B operands
     CUtensorMap map_panel_rows, map_panel_box;   // the panel as K-major A (dhidden) and as MN-major A (dW)
+    CUtensorMap map_panel_store;                 // the panel in 32 x 64 boxes: what an epilogue warp stores at a time
     if ((rc = make_map(&map_h_rows, hidden, T, d, ldh, BM)) != PODS_OK) return rc;
     if ((rc = make_map(&map_w_rows, W, V, d, ldw, BN)) != PODS_OK) return rc;
     if ((rc = make_map(&map_w_box, W, V, d, ldw, 64)) != PODS_OK) return rc;
     if ((rc = make_map(&map_h_box, hidden, T, d, ldh, 64)) != PODS_OK) return rc;
     if ((rc = make_map(&map_panel_rows, panel, l.rows_padded, l.ldp, l.ldp, BM)) != PODS_OK) return rc;
     if ((rc = make_map(&map_panel_box, panel, l.rows_padded, l.ldp, l.ldp, 64)) != PODS_OK) return rc;
-    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_dlogits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    if ((rc = make_map(&map_panel_store, panel, l.rows_padded, l.ldp, l.ldp, 32)) != PODS_OK) return rc;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_dlogits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDlogitsSmemBytes));
 
     for (int p = 0; p < l.n_panels; ++p) {
         const int tile0 = p * l.tiles_per_panel;
@@ -508,13 +575,12 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
         da.n_row_blocks = pp.n_row_blocks;
         da.tile0 = tile0;
         da.n_col_tiles = n_tiles;
-        da.tiles_per_part = pp.tiles_per_part;
-        da.n_items = (int64_t)pp.n_parts * pp.n_row_blocks;
+        da.group_rows = pp.n_row_blocks < 16 ? pp.n_row_blocks : 16;
+        da.n_items = (int64_t)n_tiles * pp.n_row_blocks;
         da.grad = grad;
-        da.panel = panel;
         da.ldp = l.ldp;
         da.status = status;
-        lm_head_dlogits_kernel<<<pp.grid, kThreads, kSmemBytes, s>>>(map_h_rows, map_w_rows, da);
+        lm_head_dlogits_kernel<<<(int)(da.n_items < sms ? da.n_items : sms), kDlogitsThreads, kDlogitsSmemBytes, s>>>(map_h_rows, map_w_rows, map_panel_store, da);
         PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
 
         GemmArgs gh;                             // dhidden[T, d] (+)= panel[T, cols] . W[tile0 * 256 + (0 .. cols), d]
