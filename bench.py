@@ -394,6 +394,107 @@ def time_lm_head(dev, T=16384, V=151936, d=2048, seconds=2.0):
             "logits_bytes_not_written": 2 * T * V, "device_status_word": binding.read_status(status)}
 
 
+def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0):
+    """grpo_loss_from_hidden (objective + dhidden + dW, neither logits nor their gradient stored in full) on one
+    chunk at the Qwen vocabulary.  The call issues 8 T V d flop (the logits are formed twice) of which 6 T V d are
+    the three products the mathematics needs; both rates are given against the measured bf16 GEMM rates.  Beside
+    it, for context: the same results from stored logits - the framework's library GEMMs for the three products
+    around this library's grpo_loss_chunk - with the extra device memory each way needs."""
+    from paper_2504_13818_b200 import binding
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4321)
+    hidden = torch.randn((T, d), generator=gen, device=dev).to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=gen, device=dev) * (3.0 / d ** 0.5)).to(torch.bfloat16)
+    tokens = torch.randint(0, V, (T,), generator=gen, device=dev, dtype=torch.int32)
+    M = 64
+    cu = torch.linspace(0, T, M + 1, device=dev).to(torch.int64)
+    adv = torch.randn(M, generator=gen, device=dev)
+    sw = binding.grpo_seq_weights(None, cu)
+    status = binding.new_status(dev)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    ws0 = torch.empty(binding.grpo_logp_from_hidden_workspace_bytes(T, V, d), dtype=torch.uint8, device=dev)
+    binding.grpo_logp_from_hidden(hidden, W, tokens, logp=logp, workspace=ws0, status=status)
+    old = logp + 0.05 * torch.randn(T, generator=gen, device=dev)
+    ref = logp + 0.1 * torch.randn(T, generator=gen, device=dev)
+    del ws0
+    loss_acc = torch.zeros(1, dtype=torch.float64, device=dev)
+    dW = torch.zeros((V, d), dtype=torch.float32, device=dev)
+    dh = torch.empty((T, d), dtype=torch.float32, device=dev)
+    ws = torch.empty(binding.grpo_loss_from_hidden_workspace_bytes(T, V, d), dtype=torch.uint8, device=dev)
+
+    def launch():
+        binding.grpo_loss_from_hidden(hidden, W, tokens, old, ref, adv, sw, cu, 0, None, 0.2, 0.04, loss_acc, dW,
+                                      logp=logp, dhidden=dh, workspace=ws, status=status)
+
+    def timed(fn, reps):
+        out = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1))
+        return out
+
+    for _ in range(2):
+        launch()
+    torch.cuda.synchronize()
+    alone = timed(launch, 5)
+    n = max(5, int(seconds * 1e3 / min(alone)))
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        launch()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_loop = e0.elapsed_time(e1) / n
+    status_word = binding.read_status(status)
+    fused_bytes = ws.numel()
+    del ws
+
+    # the same from stored logits: library GEMMs + this library's loss kernel (context, not the product)
+    logits = torch.empty((T, V), dtype=torch.bfloat16, device=dev)
+    ws2 = torch.empty(binding.grpo_loss_chunk_workspace_bytes(T), dtype=torch.uint8, device=dev)
+    dh16 = torch.empty((T, d), dtype=torch.bfloat16, device=dev)
+    dW16 = torch.empty((V, d), dtype=torch.bfloat16, device=dev)
+
+    def unfused():
+        torch.matmul(hidden, W.t(), out=logits)
+        binding.grpo_loss_chunk(logits, tokens, old, ref, adv, sw, cu, 0, None, 0.2, 0.04, loss_acc, logp, logits, ws2,
+                                status=status)
+        torch.matmul(logits, W, out=dh16)
+        torch.matmul(logits.t(), hidden, out=dW16)
+
+    for _ in range(2):
+        unfused()
+    torch.cuda.synchronize()
+    unfused_ms = timed(unfused, 5)
+    stored_bytes = logits.numel() * 2 + ws2.numel()
+
+    flop_useful, flop_issued = 6.0 * T * V * d, 8.0 * T * V * d
+    peaks = measured_peaks()
+    burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
+    return {"kernels": ["lm_head_stats_kernel", "lm_head_dlogits_kernel", "lm_head_grad_gemm_kernel<0>",
+                        "lm_head_grad_gemm_kernel<1>"], "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
+            "ms_alone_best": min(alone), "ms_alone_all": alone,
+            "issued_alone": flop_issued / min(alone) / 1e9, "useful_alone": flop_useful / min(alone) / 1e9,
+            "peak_burst": burst, "frac_issued_alone_of_burst": flop_issued / min(alone) / 1e9 / burst,
+            "ms_loop": ms_loop, "launches": n, "issued_loop": flop_issued / ms_loop / 1e9,
+            "useful_loop": flop_useful / ms_loop / 1e9, "peak_sustained": sustained,
+            "frac_issued_loop_of_sustained": flop_issued / ms_loop / 1e9 / sustained,
+            "frac_useful_loop_of_sustained": flop_useful / ms_loop / 1e9 / sustained,
+            "peak_kind": "of measured" if peaks else "of fallback",
+            "sm_mhz_median": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
+            "tokens_per_s_loop": T / (ms_loop * 1e-3), "workspace_bytes": fused_bytes,
+            "from_stored_logits": {"what": "library GEMMs (logits, dhidden, dW; bf16 outputs) around grpo_loss_chunk in place",
+                                   "ms_best": min(unfused_ms), "ms_all": unfused_ms, "extra_bytes": stored_bytes},
+            "device_status_word": status_word}
+
+
 def cpu_baseline(batch, budget_rows=None):
     """The CPU checker, as it stands, on a bounded sample of the same batch (rank 0, N=1 only)."""
     import oracle
@@ -512,6 +613,7 @@ def run_ours(args):
         out["pods_select"] = [time_select(nm, dev, 20, 3) for nm in ("c3_select_mixed", "c4_select_ties")]
     if rank == 0 and world == 1 and not args.no_lm_head:
         out["lm_head"] = time_lm_head(dev)
+        out["lm_head_loss"] = time_lm_head_loss(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(batch)
     if rank == 0:
