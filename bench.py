@@ -394,7 +394,7 @@ def time_lm_head(dev, T=16384, V=151936, d=2048, seconds=2.0):
             "logits_bytes_not_written": 2 * T * V, "device_status_word": binding.read_status(status)}
 
 
-def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0):
+def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0, compare=True):
     """grpo_loss_from_hidden (objective + dhidden + dW, neither logits nor their gradient stored in full) on one
     chunk at the Qwen vocabulary.  The call issues 8 T V d flop (the logits are formed twice) of which 6 T V d are
     the three products the mathematics needs; both rates are given against the measured bf16 GEMM rates.  Beside
@@ -456,6 +456,25 @@ def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0):
     fused_bytes = ws.numel()
     del ws
 
+    flop_useful, flop_issued = 6.0 * T * V * d, 8.0 * T * V * d
+    peaks = measured_peaks()
+    burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
+    out = {"kernels": ["lm_head_stats_kernel", "lm_head_dlogits_kernel", "lm_head_grad_gemm_kernel<0>",
+                       "lm_head_grad_gemm_kernel<1>"], "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
+           "ms_alone_best": min(alone), "ms_alone_all": alone,
+           "issued_alone": flop_issued / min(alone) / 1e9, "useful_alone": flop_useful / min(alone) / 1e9,
+           "peak_burst": burst, "frac_issued_alone_of_burst": flop_issued / min(alone) / 1e9 / burst,
+           "ms_loop": ms_loop, "launches": n, "issued_loop": flop_issued / ms_loop / 1e9,
+           "useful_loop": flop_useful / ms_loop / 1e9, "peak_sustained": sustained,
+           "frac_issued_loop_of_sustained": flop_issued / ms_loop / 1e9 / sustained,
+           "frac_useful_loop_of_sustained": flop_useful / ms_loop / 1e9 / sustained,
+           "peak_kind": "of measured" if peaks else "of fallback",
+           "sm_mhz_median": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
+           "tokens_per_s_loop": T / (ms_loop * 1e-3), "workspace_bytes": fused_bytes,
+           "device_status_word": status_word}
+    if not compare:
+        return out
+
     # the same from stored logits: library GEMMs + this library's loss kernel (context, not the product)
     logits = torch.empty((T, V), dtype=torch.bfloat16, device=dev)
     ws2 = torch.empty(binding.grpo_loss_chunk_workspace_bytes(T), dtype=torch.uint8, device=dev)
@@ -475,24 +494,9 @@ def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0):
     unfused_ms = timed(unfused, 5)
     stored_bytes = logits.numel() * 2 + ws2.numel()
 
-    flop_useful, flop_issued = 6.0 * T * V * d, 8.0 * T * V * d
-    peaks = measured_peaks()
-    burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
-    return {"kernels": ["lm_head_stats_kernel", "lm_head_dlogits_kernel", "lm_head_grad_gemm_kernel<0>",
-                        "lm_head_grad_gemm_kernel<1>"], "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
-            "ms_alone_best": min(alone), "ms_alone_all": alone,
-            "issued_alone": flop_issued / min(alone) / 1e9, "useful_alone": flop_useful / min(alone) / 1e9,
-            "peak_burst": burst, "frac_issued_alone_of_burst": flop_issued / min(alone) / 1e9 / burst,
-            "ms_loop": ms_loop, "launches": n, "issued_loop": flop_issued / ms_loop / 1e9,
-            "useful_loop": flop_useful / ms_loop / 1e9, "peak_sustained": sustained,
-            "frac_issued_loop_of_sustained": flop_issued / ms_loop / 1e9 / sustained,
-            "frac_useful_loop_of_sustained": flop_useful / ms_loop / 1e9 / sustained,
-            "peak_kind": "of measured" if peaks else "of fallback",
-            "sm_mhz_median": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
-            "tokens_per_s_loop": T / (ms_loop * 1e-3), "workspace_bytes": fused_bytes,
-            "from_stored_logits": {"what": "library GEMMs (logits, dhidden, dW; bf16 outputs) around grpo_loss_chunk in place",
-                                   "ms_best": min(unfused_ms), "ms_all": unfused_ms, "extra_bytes": stored_bytes},
-            "device_status_word": status_word}
+    out["from_stored_logits"] = {"what": "library GEMMs (logits, dhidden, dW; bf16 outputs) around grpo_loss_chunk in place",
+                                 "ms_best": min(unfused_ms), "ms_all": unfused_ms, "extra_bytes": stored_bytes}
+    return out
 
 
 def cpu_baseline(batch, budget_rows=None):

@@ -415,6 +415,8 @@ def grpo_loss_from_hidden(hidden, W, tokens, old_logp, ref_logp, adv, seq_weight
     _numel(adv, M, "adv")
     _numel(seq_weight, M, "seq_weight")
     _numel(loss_acc, 1, "loss_acc")
+    _require(isinstance(dhidden, torch.Tensor) and tuple(dhidden.shape) == (T, d), "dhidden must have the shape [%d, %d]" % (T, d))
+    _require(isinstance(dW, torch.Tensor) and tuple(dW.shape) == (V, d), "dW must have the shape [%d, %d]" % (V, d))
     need = grpo_loss_from_hidden_workspace_bytes(T, V, d)
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)

@@ -133,3 +133,50 @@ def test_binding_checks_every_buffer_length_before_the_call():
         binding.pods_select_into(r, n + 1, idx, torch.zeros((G, m)))
     with pytest.raises(binding.PodsError, match="seq_weight must hold"):
         binding.grpo_seq_weights(None, torch.zeros(M + 1, dtype=torch.int64), out=torch.zeros(M + 2, dtype=torch.float64))
+
+
+def test_loss_from_hidden_checks_sizes_on_the_host():
+    """grpo_loss_from_hidden: the library refuses impossible sizes before launching, the binding refuses short or
+    mis-shaped buffers before marshalling, and the panel limit is a process-wide setting with a floor."""
+    import pytest
+    import torch
+    lib = binding.load()
+    fake = C.c_void_p(256)
+
+    def call(T=4, V=16, d=8, ldh=8, ldw=8, lddh=8, lddw=8, beta=0.0, ref=None, ws=None, ws_bytes=0):
+        return lib.grpo_loss_from_hidden(fake, ldh, fake, ldw, fake, fake, ref, fake, fake, fake, 1, 0, None, T, V, d,
+                                         0.2, beta, 1.0, fake, fake, fake, lddh, fake, lddw, ws, ws_bytes, None, None)
+
+    assert call(d=12) == 1 and call(ldh=4) == 1 and call(lddw=6) == 1 and call(V=0) == 1     # sizes
+    assert call(beta=0.04) == 1                                                              # beta != 0 needs ref_logp
+    assert call() == 3                                                                       # no workspace
+    assert call(T=0) == 0                                                                    # empty chunk
+    need = lib.grpo_loss_from_hidden_workspace_bytes(300, 1000, 64)
+    assert need >= 384 * 1024 * 2                       # at least the panel of one launch: 384 rows x 4 tiles, bf16
+    default = lib.pods_set_loss_from_hidden_panel_bytes(1)
+    assert default == 512 << 20
+    assert lib.grpo_loss_from_hidden_workspace_bytes(300, 1000, 64) < need        # one tile per panel now
+    assert lib.pods_set_loss_from_hidden_panel_bytes(default) == 65536            # the floor
+    assert lib.grpo_loss_from_hidden_workspace_bytes(300, 1000, 64) == need
+
+    T, V, d, M = 12, 40, 16, 3
+    def args(**over):
+        a = dict(hidden=torch.zeros((T, d), dtype=torch.bfloat16), W=torch.zeros((V, d), dtype=torch.bfloat16),
+                 tokens=torch.zeros(T, dtype=torch.int32), old_logp=torch.zeros(T), ref_logp=torch.zeros(T),
+                 adv=torch.zeros(M), seq_weight=torch.zeros(M, dtype=torch.float64),
+                 cu_seqlens=torch.zeros(M + 1, dtype=torch.int64), row0=0, mask=torch.ones(T, dtype=torch.uint8),
+                 eps=0.2, beta=0.04, loss_acc=torch.zeros(1, dtype=torch.float64), dW=torch.zeros((V, d)),
+                 logp=torch.zeros(T), dhidden=torch.zeros((T, d)))
+        a.update(over)
+        return a
+
+    wrong = {"W": torch.zeros((V, d + 8), dtype=torch.bfloat16), "tokens": torch.zeros(T - 1, dtype=torch.int32),
+             "old_logp": torch.zeros(T + 1), "ref_logp": torch.zeros(1), "mask": torch.ones(T - 2, dtype=torch.uint8),
+             "logp": torch.zeros(T - 1), "adv": torch.zeros(M + 1), "seq_weight": torch.zeros(M - 1, dtype=torch.float64),
+             "loss_acc": torch.zeros(2, dtype=torch.float64), "dW": torch.zeros((V - 1, d)),
+             "dhidden": torch.zeros((T, d + 1)), "workspace": torch.zeros(8, dtype=torch.uint8)}
+    for name, bad in wrong.items():
+        with pytest.raises(binding.PodsError, match="must hold|must have"):
+            binding.grpo_loss_from_hidden(**args(**{name: bad}))
+    with pytest.raises(binding.PodsError, match="CUDA"):           # every length right: only the device is wrong
+        binding.grpo_loss_from_hidden(**args())

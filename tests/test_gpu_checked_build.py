@@ -15,6 +15,8 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SUBSET = ["tests/test_gpu_select.py", "tests/test_gpu_compact.py", "tests/test_gpu_accumulation.py",
           "tests/test_gpu_lm_head.py::test_logp_against_the_oracle_on_all_rows",
+          "tests/test_gpu_lm_head_loss.py::test_loss_and_gradients_against_the_oracle",
+          "tests/test_gpu_lm_head_loss.py::test_several_panels_accumulate_to_the_same_result",
           "tests/test_gpu_loss.py::test_config1_whole_path_values",
           "tests/test_gpu_loss.py::test_vocab_sizes_span_tiles_and_ragged_tails",
           "tests/test_gpu_loss.py::test_cluster_path_vocab_sizes",
