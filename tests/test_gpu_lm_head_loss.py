@@ -3,11 +3,13 @@ gradient with respect to hidden and W, the [T,V] logits and their gradient never
 
 Tolerances.  logp abs <= 1e-3 and the loss as everywhere else.  The gradients are sums of products
 dlogits[t,v] W[v,j] (over v) and dlogits[t,v] hidden[t,j] (over t) in which the kernel rounds dlogits to bf16 - as the
-unfused path's stored gradient is - so every term carries a relative error of at most 2^-9; the fp32 evaluation of the
-softmax (logits accumulated in fp32 over d terms, the fp32 log-sum-exp) and the fp32 accumulation of the sums add a
-few 1e-5 relative to the terms.  Hence, element by element,
-    |gpu - oracle| <= 2^-8 * sum |dlogits| |W|      (dhidden)        2^-8 * sum |dlogits| |hidden|      (dW),
-the sums of magnitudes coming from the oracle.  The bound assumes that no row's factor g_t is itself a cancellation
+unfused path's stored gradient is - so every term carries a relative error of at most 2^-8, the unit roundoff of bf16
+(reached by values just above a power of two); the fp32 evaluation of the softmax (logits accumulated in fp32 over d
+terms, the fp32 log-sum-exp) and the fp32 accumulation of the sums add a few 1e-5 relative to the terms, for which
+2^-12 is allowed.  Hence, element by element,
+    |gpu - oracle| <= (2^-8 + 2^-12) * sum |dlogits| |W|   (dhidden)      (2^-8 + 2^-12) * sum |dlogits| |hidden|   (dW),
+the sums of magnitudes coming from the oracle; where one term dominates a sum the measured error comes within a few
+per cent of 2^-8, as it must.  The bound assumes that no row's factor g_t is itself a cancellation
 (reading of the dlogits tolerance for the unfused kernel); the inputs are drawn so that there is none, which is asserted.
 """
 import numpy as np
@@ -21,7 +23,7 @@ from parity import LOGP_ATOL, LOSS_RTOL, record
 
 pytestmark = pytest.mark.gpu
 
-GRAD_RTOL = 2.0 ** -8
+GRAD_RTOL = 2.0 ** -8 + 2.0 ** -12
 EPS, BETA = 0.2, 0.04
 
 
