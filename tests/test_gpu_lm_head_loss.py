@@ -203,3 +203,71 @@ def test_qwen_vocabulary_at_d_2048():
         binding.set_loss_from_hidden_panel_bytes(before)
     _compare("grpo_loss_from_hidden T=512 V=151936 d=2048", got, want, c)
     assert abs(got["loss"] - want["loss"]) <= LOSS_RTOL * max(abs(want["loss"]), np.abs(want["ell"]).mean() / 1e3)
+
+
+@pytest.mark.skipif(not torch.cuda.is_available() or torch.cuda.get_device_properties(0).total_memory < 20e9,
+                    reason="needs a few GB of device memory")
+def test_bench_shape_on_sampled_rows_and_by_identities():
+    """T = 16384, V = 151936, d = 2048: the call bench.py times (ten panels).  The oracle takes sampled rows one block
+    at a time: their log-probs and rows of dhidden (a row of dhidden depends on that row alone).  dW as a whole is tied
+    to dhidden by two identities that hold at any size:
+      <dW, W> = sum_{t,v} dlogits[t,v] logits[t,v] = <dhidden, hidden>     and     sum_v dW[v, :] = 0
+    (every row of dlogits sums to zero), each up to the rounding of dlogits to bf16."""
+    T, V, d, M = 16384, 151936, 2048, 64
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(77)
+    hidden = torch.randn((T, d), generator=gen, device=dev).to(torch.bfloat16)
+    W = (torch.randn((V, d), generator=gen, device=dev) * (3.0 / d ** 0.5)).to(torch.bfloat16)
+    tokens = torch.randint(0, V, (T,), generator=gen, device=dev, dtype=torch.int32)
+    # old / ref: the framework's stock log-softmax of the same product plus noise - it only shapes the inputs
+    base = torch.empty(T, device=dev)
+    for lo in range(0, T, 2048):
+        x = (hidden[lo:lo + 2048] @ W.t()).float()
+        base[lo:lo + 2048] = torch.log_softmax(x, dim=-1).gather(1, tokens[lo:lo + 2048].long()[:, None])[:, 0]
+        del x
+    noise = 0.1 * torch.randn(T, generator=gen, device=dev)
+    old = base + 0.15 * torch.randn(T, generator=gen, device=dev)
+    ref = base + torch.sign(noise) * (0.02 + noise.abs())
+    rng = np.random.default_rng(77)
+    cu_h = np.concatenate([[0], np.sort(rng.choice(np.arange(1, T), size=M - 1, replace=False)), [T]]).astype(np.int64)
+    adv_h = rng.normal(size=M)
+    adv_h = (np.sign(adv_h) * (0.2 + np.abs(adv_h))).astype(np.float32)
+    mask_h = np.ones(T, np.uint8)
+    mask_h[rng.integers(0, T, 200)] = 0
+    cu, adv, mask = torch.from_numpy(cu_h).to(dev), torch.from_numpy(adv_h).to(dev), torch.from_numpy(mask_h).to(dev)
+    sw = binding.grpo_seq_weights(mask, cu)
+    loss_acc = torch.zeros(1, dtype=torch.float64, device=dev)
+    dW = torch.zeros((V, d), dtype=torch.float32, device=dev)
+    status = binding.new_status()
+    logp, dh = binding.grpo_loss_from_hidden(hidden, W, tokens, old, ref, adv, sw, cu, 0, mask, EPS, BETA, loss_acc, dW,
+                                             status=status)
+    torch.cuda.synchronize()
+    assert binding.read_status(status) == 0
+
+    rows = np.unique(np.concatenate([[0, 127, 128, T - 1], cu_h[1:5] - 1, cu_h[1:5], np.flatnonzero(mask_h == 0)[:4],
+                                     rng.integers(0, T, 80)]))
+    seq = oracle.seq_of_rows(cu_h)
+    want = lm_head.loss_grad_from_hidden(hidden[rows].view(torch.uint16).cpu().numpy(), W.view(torch.uint16).cpu().numpy(),
+                                         tokens.cpu().numpy()[rows], old.cpu().numpy()[rows], ref.cpu().numpy()[rows],
+                                         adv_h, oracle.seq_weights(mask_h, cu_h), seq[rows], mask_h[rows], EPS, BETA,
+                                         block_rows=32)
+    logp_err = float(np.abs(logp.cpu().numpy()[rows] - want["logp"]).max())
+    got = dh[rows].cpu().numpy().astype(np.float64)
+    dh_ratio = float((np.abs(got - want["dhidden"]) / (want["abs_dhidden"] + 1e-30)).max())
+    # the identities, in fp64 on the device
+    dW64, W64 = dW.double(), W.double()
+    lhs = float((dW64 * W64).sum())
+    rhs = float((dh.double() * hidden.double()).sum())
+    scale = float((dW64.abs() * W64.abs()).sum() + (dh.double().abs() * hidden.double().abs()).sum())
+    col = dW64.sum(dim=0)
+    col_ratio = float((col.abs() / dW64.abs().sum(dim=0)).max())
+    record("grpo_loss_from_hidden T=%d V=%d d=%d (%d sampled rows)" % (T, V, d, len(rows)), logp_abs=logp_err,
+           dhidden_over_term_sum=dh_ratio, inner_product_identity=abs(lhs - rhs) / scale, dW_column_sum_ratio=col_ratio,
+           bound=GRAD_RTOL)
+    assert logp_err <= LOGP_ATOL
+    assert dh_ratio <= GRAD_RTOL
+    assert (got[want["abs_dhidden"].max(axis=1) == 0] == 0).all()          # masked rows among the sample
+    assert abs(lhs - rhs) <= GRAD_RTOL * scale
+    assert col_ratio <= GRAD_RTOL
+    assert torch.isfinite(dW).all() and torch.isfinite(dh).all()
