@@ -188,6 +188,121 @@ __device__ __forceinline__ bool drain_loads(Barriers& bar, int64_t loads) {
     return ok;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// CTA pairs (a cluster of two CTAs on the two SMs of a TPC, tcgen05 cta_group::2): the pair computes one
+// 256 x 256 tile; each CTA loads its own 128 rows of A and HALF of B (128 of the 256 columns), the leader (cluster
+// rank 0) issues the MMAs for both, each CTA's tensor memory receives its own 128 rows of the accumulator.  Per
+// contraction block a CTA then takes 32 KB from L2 instead of 48 KB, and the ring holds six stages instead of four.
+// Barriers live at the same shared-memory offsets in both CTAs.  No load is multicast: every CTA issues its own loads
+// into its own shared memory; only the completion is counted on the LEADER's barrier.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairStageBytesA = BM * BK * 2, kPairStageBytesB = (BN / 2) * BK * 2;
+constexpr uint32_t kPairStageBytes = kPairStageBytesA + kPairStageBytesB;          // per CTA
+constexpr size_t kPairSmemBytes = 1024 + (size_t)kPairStages * kPairStageBytes + 256;
+
+struct PairBarriers {
+    unsigned long long full[kPairStages];      // leader's: both CTAs' loads of the stage have landed
+    unsigned long long empty[kPairStages];     // each CTA's own: the stage has been consumed (signalled in both CTAs)
+    unsigned long long acc_full[kAccumulators];    // each CTA's own: the accumulator is complete (signalled in both)
+    unsigned long long acc_empty[kAccumulators];   // leader's: the epilogue warps of BOTH CTAs have read it
+    uint32_t tmem_base;
+    uint32_t pad;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The shared::cluster address of the same shared-memory location in the pair's leader (cluster rank 0).
+__device__ __forceinline__ uint32_t leader_addr(const void* p) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(smem_u32(p)));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_leader(const void* bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_addr(bar)) : "memory");
+}
+// A box into THIS CTA's shared memory; the bytes are counted on the LEADER's barrier at the same offset.
+__device__ __forceinline__ void tma_load_tile_pair(void* dst, const CUtensorMap* map, int x, int y, const void* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(leader_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_tile_pair_hint(void* dst, const CUtensorMap* map, int x, int y, const void* bar,
+                                                        uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(leader_addr(bar)), "l"(policy) : "memory");
+}
+// Instruction descriptor of the pair's MMA: M = 256 (128 rows in each CTA), N = 256.
+__host__ __device__ constexpr uint32_t instr_desc_pair(bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+}
+__device__ __forceinline__ void umma_pair(uint32_t tmem_acc, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_acc), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this offset in BOTH CTAs of the pair once every MMA issued so far has completed.
+__device__ __forceinline__ void umma_commit_pair(void* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+// Both CTAs of the pair call these with the same warp (warp 1).
+__device__ __forceinline__ void tmem_alloc_all_pair(uint32_t* slot) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free_all_pair(uint32_t tmem_base) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+// Barriers initialised (both CTAs initialise their own copies), tensor memory allocated, and the whole PAIR in step:
+// no CTA may signal its partner's barriers before they exist.
+__device__ __forceinline__ uint32_t pair_setup(PairBarriers& bar, int warp, uint32_t epilogue_warps_per_cta) {
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&bar.full[s], 1); mbar_init(&bar.empty[s], 1); }
+        for (int b = 0; b < kAccumulators; ++b) {
+            mbar_init(&bar.acc_full[b], 1);
+            mbar_init(&bar.acc_empty[b], 2 * epilogue_warps_per_cta);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_all_pair(&bar.tmem_base);
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tcgen05_fence_after();
+    return bar.tmem_base;
+}
+// Neither CTA may leave (its shared memory and barriers are the partner's too) before both are done.
+__device__ __forceinline__ void pair_teardown(uint32_t tmem_base, int warp) {
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_free_all_pair(tmem_base);
+    }
+}
+// The last use of each stage's full barrier (leader only): every load of BOTH CTAs has landed.
+__device__ __forceinline__ bool drain_loads_pair(PairBarriers& bar, int64_t loads) {
+    bool ok = true;
+    for (int s = 0; s < kPairStages; ++s) {
+        const int64_t uses = loads > s ? (loads - s + kPairStages - 1) / kPairStages : 0;
+        if (uses > 0 && !mbar_wait(&bar.full[s], (uint32_t)((uses - 1) & 1), false)) ok = false;
+    }
+    return ok;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);

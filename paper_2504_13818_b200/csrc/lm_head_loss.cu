@@ -10,14 +10,17 @@
 //   3. lm_head_dlogits_kernel: the panel's logits AGAIN on the tensor cores (same pipeline as pass 1), and in the
 //      epilogue dlogits = g_t ([v == token] - 2^(x log2e - lse log2e)) rounded to bf16 into the panel buffer
 //      [rows, panel columns] - the only place a piece of the [T,V] gradient ever exists;
-//   4. lm_head_grad_gemm_kernel<false>: dhidden[T,d] (+)= panel[T, cols] . W[cols, d]
-//   5. lm_head_grad_gemm_kernel<true>:  dW[cols, d] += panel^T[cols, T] . hidden[T, d]
+//   4. lm_head_grad_gemm_pair_kernel<false>: dhidden[T,d] (+)= panel[T, cols] . W[cols, d]
+//   5. lm_head_grad_gemm_pair_kernel<true>:  dW[cols, d] += panel^T[cols, T] . hidden[T, d]
 //      both with tcgen05.mma reading the operands whose contraction index is NOT contiguous in memory (W and hidden
 //      by rows of d, the panel by rows of vocabulary entries for step 5) as MN-major shared-memory tiles, so
 //      no transposed copy of anything is made.
 // Roles, barriers and bounded waits are those of the statistics kernel: a TMA producer warp, one thread issuing
 // the MMAs into one of two 256-column accumulators in tensor memory, four epilogue warps (one tile row per
-// thread; eight warps, half a row per thread, where the epilogue forms the gradient).  All loads are plain (never multicast) TMA loads of this GPU's own memory.
+// thread; eight warps, half a row per thread, where the epilogue forms the gradient).  Kernels 3-5 run as PAIRS of
+// CTAs (cta_group::2): a pair shares one 256 x 256 tile, each CTA loading its rows of A and half of B, which cuts the
+// bytes a CTA takes from L2 per contraction block from 48 KB to 32 KB and deepens the ring from four to six stages.
+// All loads are plain (never multicast) TMA loads of this GPU's own memory into the loading CTA's own shared memory.
 
 #include "grpo_loss_common.cuh"
 #include "lm_head_common.cuh"
@@ -87,13 +90,14 @@ lm_head_row_terms_kernel(const TermsArgs a) {
 // ------------------------------------------------------------------------------------------------------
 struct DlogitsArgs {
     int32_t V, d;
-    int32_t n_row_blocks;
+    int32_t n_row_blocks;        // PAIRS of 128-row blocks (what tile_of counts)
+    int32_t n_blocks128;         // 128-row blocks: the panel and `grad` have n_blocks128 * 128 rows
     int32_t tile0;               // first 256-column tile of the panel, counted over the whole vocabulary
     int32_t n_col_tiles;         // tiles of this panel
     int32_t group_rows;          // row blocks per group of the tile order (see tile_of)
     int64_t n_items;             // tiles of the panel: column tiles x row blocks
-    const RowGrad* grad;         // [n_row_blocks * 128]
-    int64_t ldp;                 // row pitch of the panel (bf16 [n_row_blocks * 128, ldp]), >= n_col_tiles * 256
+    const RowGrad* grad;         // [n_blocks128 * 128]
+    int64_t ldp;                 // row pitch of the panel (bf16 [n_blocks128 * 128, ldp]), >= n_col_tiles * 256
     uint32_t* status;
 };
 
@@ -126,18 +130,22 @@ constexpr int kDlogitsThreads = 64 + 8 * 32;
 // sends them off as one bulk tensor store.  Stored straight from registers (16 bytes per lane and instruction, every
 // lane another line) the same data cost 1.5 ms of 7.7 per 16384 rows.
 constexpr uint32_t kStagingBytesPerWarp = 32 * 128;
-constexpr size_t kDlogitsSmemBytes = 1024 + (size_t)kStages * kStageBytes + 8 * kStagingBytesPerWarp + 256;
+constexpr size_t kDlogitsSmemBytes = 1024 + (size_t)kPairStages * kPairStageBytes + 8 * kStagingBytesPerWarp + 256;
 
-__global__ void __launch_bounds__(kDlogitsThreads, 1)
+// CTA pairs (see lm_head_common.cuh): an item is a 256 x 256 tile of logits, CTA r of the pair holds rows 128 r ..
+// of it and loads columns 128 r .. of W's tile; n_row_blocks, group_rows and tile_of count PAIRS of 128-row blocks.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDlogitsThreads, 1)
 lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_panel, const DlogitsArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* const tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* const staging = tiles + (size_t)kStages * kStageBytes;        // 1024-byte aligned, 4 KB per warp
-    Barriers& bar = *reinterpret_cast<Barriers*>(staging + 8 * kStagingBytesPerWarp);
+    unsigned char* const staging = tiles + (size_t)kPairStages * kPairStageBytes;    // 1024-byte aligned, 4 KB per warp
+    PairBarriers& bar = *reinterpret_cast<PairBarriers*>(staging + 8 * kStagingBytesPerWarp);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_blocks = (a.d + BK - 1) / BK;
-    const uint32_t tmem_base = pipeline_setup(bar, warp, 8);
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t tmem_base = pair_setup(bar, warp, 8);
+    const int64_t first = blockIdx.x >> 1, stride = gridDim.x >> 1;
     bool timed_out = false;
 
     if (warp == 0) {
@@ -145,31 +153,32 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
             int stage = 0;
             uint32_t phase = 0;
             int64_t loads = 0;
-            for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+            for (int64_t item = first; item < a.n_items; item += stride) {
                 int ct, rb;
                 tile_of(a, item, &ct, &rb);
                 {
                     for (int kb = 0; kb < k_blocks; ++kb) {
                         if (!mbar_wait(&bar.empty[stage], phase ^ 1u, timed_out)) timed_out = true;
-                        unsigned char* sa = tiles + (size_t)stage * kStageBytes;
-                        mbar_expect_tx(&bar.full[stage], kStageBytes);
-                        tma_load_tile(sa, &map_hidden, kb * BK, rb * BM, &bar.full[stage]);
-                        tma_load_tile(sa + kStageBytesA, &map_w, kb * BK, (a.tile0 + ct) * BN, &bar.full[stage]);
+                        unsigned char* sa = tiles + (size_t)stage * kPairStageBytes;
+                        if (rank == 0) mbar_expect_tx(&bar.full[stage], 2 * kPairStageBytes);
+                        tma_load_tile_pair(sa, &map_hidden, kb * BK, (2 * rb + (int)rank) * BM, &bar.full[stage]);
+                        tma_load_tile_pair(sa + kPairStageBytesA, &map_w, kb * BK,
+                                           (a.tile0 + ct) * BN + (int)rank * (BN / 2), &bar.full[stage]);
                         ++loads;
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
-            if (!drain_loads(bar, loads)) timed_out = true;
+            if (rank == 0 && !drain_loads_pair(bar, loads)) timed_out = true;
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
             uint32_t acc_phase = 0;
-            for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+            for (int64_t item = first; item < a.n_items; item += stride) {
                 {
                     if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
                     tcgen05_fence_after();
@@ -177,16 +186,16 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
                     for (int kb = 0; kb < k_blocks; ++kb) {
                         if (!mbar_wait(&bar.full[stage], phase, timed_out)) timed_out = true;
                         tcgen05_fence_after();
-                        const uint32_t sa = smem_u32(tiles + (size_t)stage * kStageBytes);
-                        const uint64_t da = smem_desc_k_major(sa), db = smem_desc_k_major(sa + kStageBytesA);
+                        const uint32_t sa = smem_u32(tiles + (size_t)stage * kPairStageBytes);
+                        const uint64_t da = smem_desc_k_major(sa), db = smem_desc_k_major(sa + kPairStageBytesA);
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; ++k)
-                            umma(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 >> 4), db + (uint64_t)(k * UMMA_K * 2 >> 4),
-                                 instr_desc(false, false), (kb | k) != 0 ? 1u : 0u);
-                        umma_commit(&bar.empty[stage]);
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                            umma_pair(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 >> 4), db + (uint64_t)(k * UMMA_K * 2 >> 4),
+                                      instr_desc_pair(false, false), (kb | k) != 0 ? 1u : 0u);
+                        umma_commit_pair(&bar.empty[stage]);
+                        if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                     }
-                    umma_commit(&bar.acc_full[acc]);
+                    umma_commit_pair(&bar.acc_full[acc]);
                     if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
                 }
             }
@@ -203,11 +212,14 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
         const uint64_t stream_policy = l2_policy_evict_first();      // the panel is written once and read much later
         int acc = 0;
         uint32_t acc_phase = 0;
-        for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+        for (int64_t item = first; item < a.n_items; item += stride) {
             int ct, rb;
             tile_of(a, item, &ct, &rb);
-            const int64_t row = (int64_t)rb * BM + row_in_tile;
-            const RowGrad rg = a.grad[PODS_CLAMPED(row, (int64_t)a.n_row_blocks * BM, a.status)];
+            const int block = 2 * rb + (int)rank;                         // this CTA's 128-row block
+            const bool block_ok = block < a.n_blocks128;                  // an odd count leaves the last pair's second half empty
+            const int64_t row = (int64_t)block * BM + row_in_tile;
+            const RowGrad rg = block_ok ? a.grad[PODS_CLAMPED(row, (int64_t)a.n_blocks128 * BM, a.status)]
+                                        : RowGrad{0.0f, 0.0f, 0, 0.0f};
             const float neg_g = -rg.g;
             {
                 if (!mbar_wait(&bar.acc_full[acc], acc_phase, timed_out)) timed_out = true;
@@ -248,16 +260,16 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
                         *reinterpret_cast<uint4*>(stage_line + ((j ^ (lane & 7)) << 4)) = q[j];
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0 && PODS_INDEX_OK((int64_t)ct * BN + c0 + 63, a.ldp, a.status)) {
+                    if (lane == 0 && block_ok && PODS_INDEX_OK((int64_t)ct * BN + c0 + 63, a.ldp, a.status)) {
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
                                      ::"l"(reinterpret_cast<uint64_t>(&map_panel)), "r"(ct * BN + c0),
-                                       "r"(rb * BM + quarter * 32), "r"(smem_u32(stage_warp)), "l"(stream_policy) : "memory");
+                                       "r"(block * BM + quarter * 32), "r"(smem_u32(stage_warp)), "l"(stream_policy) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bar.acc_empty[acc]);
+                if (lane == 0) mbar_arrive_leader(&bar.acc_empty[acc]);
                 if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -265,7 +277,7 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
     // a warp's bulk stores must be complete before its shared memory goes away
     if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (timed_out && lane == 0) pods_raise(a.status, PODS_STATUS_TIMEOUT);
-    pipeline_teardown(tmem_base, warp);
+    pair_teardown(tmem_base, warp);
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -283,16 +295,22 @@ struct GemmArgs {
     uint32_t* status;
 };
 
+// By CTA pairs (cluster of two, tcgen05 cta_group::2): a pair owns a 256 x 256 tile of C.  CTA r of the pair loads
+// rows m0 + 128 r .. of A and columns n0 + 128 r .. of B, the leader issues M = 256 MMAs that read both CTAs' shared
+// memory and fill both CTAs' tensor memory, and each CTA's epilogue adds its own 128 rows into C.
 template <bool A_MN>
-__global__ void __launch_bounds__(kThreads, 1)
-lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                         const GemmArgs g) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+lm_head_grad_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                              const GemmArgs g) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* const tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Barriers& bar = *reinterpret_cast<Barriers*>(tiles + (size_t)kStages * kStageBytes);
+    PairBarriers& bar = *reinterpret_cast<PairBarriers*>(tiles + (size_t)kPairStages * kPairStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t tmem_base = pipeline_setup(bar, warp);
-    const int64_t n_tiles_total = (int64_t)g.m_tiles * g.n_tiles;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t tmem_base = pair_setup(bar, warp, 4);
+    const int m_pairs = (g.m_tiles + 1) / 2;
+    const int64_t n_tiles_total = (int64_t)m_pairs * g.n_tiles;
+    const int64_t first = blockIdx.x >> 1, stride = gridDim.x >> 1;
     bool timed_out = false;
 
     if (warp == 0) {
@@ -300,57 +318,57 @@ lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             int stage = 0;
             uint32_t phase = 0;
             int64_t loads = 0;
-            const uint64_t stream_policy = l2_policy_evict_first();  // the panel streams through; W and hidden are re-read
-            for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
-                const int m0 = (int)(tile / g.n_tiles) * BM, n0 = (int)(tile % g.n_tiles) * BN;
+            const uint64_t stream_policy = l2_policy_evict_first();
+            for (int64_t tile = first; tile < n_tiles_total; tile += stride) {
+                const int m0 = (int)(tile / g.n_tiles) * 2 * BM + (int)rank * BM;
+                const int n0 = (int)(tile % g.n_tiles) * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < g.k_blocks; ++kb) {
                     if (!mbar_wait(&bar.empty[stage], phase ^ 1u, timed_out)) timed_out = true;
-                    unsigned char* sa = tiles + (size_t)stage * kStageBytes;
-                    mbar_expect_tx(&bar.full[stage], kStageBytes);
+                    unsigned char* sa = tiles + (size_t)stage * kPairStageBytes;
+                    if (rank == 0) mbar_expect_tx(&bar.full[stage], 2 * kPairStageBytes);
                     if (A_MN) {
 #pragma unroll
                         for (int i = 0; i < BM / 64; ++i)
-                            tma_load_tile_hint(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage], stream_policy);
+                            tma_load_tile_pair_hint(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage], stream_policy);
                     } else {
-                        tma_load_tile_hint(sa, &map_a, kb * BK, m0, &bar.full[stage], stream_policy);
+                        tma_load_tile_pair_hint(sa, &map_a, kb * BK, m0, &bar.full[stage], stream_policy);
                     }
 #pragma unroll
-                    for (int i = 0; i < BN / 64; ++i)
-                        tma_load_tile(sa + kStageBytesA + i * kBoxBytes, &map_b, n0 + 64 * i, g.b_k0 + kb * BK, &bar.full[stage]);
+                    for (int i = 0; i < BN / 2 / 64; ++i)
+                        tma_load_tile_pair(sa + kPairStageBytesA + i * kBoxBytes, &map_b, n0 + 64 * i, g.b_k0 + kb * BK, &bar.full[stage]);
                     ++loads;
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!drain_loads(bar, loads)) timed_out = true;
+            if (rank == 0 && !drain_loads_pair(bar, loads)) timed_out = true;
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
             uint32_t acc_phase = 0;
-            constexpr uint32_t idesc = instr_desc(A_MN, true);
-            // 16 contraction entries further: 32 bytes along a K-major row, 16 rows of 128 bytes in an MN-major box
+            constexpr uint32_t idesc = instr_desc_pair(A_MN, true);
             constexpr uint64_t a_step = A_MN ? (uint64_t)(UMMA_K * 128 >> 4) : (uint64_t)(UMMA_K * 2 >> 4);
             constexpr uint64_t b_step = (uint64_t)(UMMA_K * 128 >> 4);
-            for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+            for (int64_t tile = first; tile < n_tiles_total; tile += stride) {
                 if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
                 tcgen05_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < g.k_blocks; ++kb) {
                     if (!mbar_wait(&bar.full[stage], phase, timed_out)) timed_out = true;
                     tcgen05_fence_after();
-                    const uint32_t sa = smem_u32(tiles + (size_t)stage * kStageBytes);
+                    const uint32_t sa = smem_u32(tiles + (size_t)stage * kPairStageBytes);
                     const uint64_t da = A_MN ? smem_desc_mn_major(sa) : smem_desc_k_major(sa);
-                    const uint64_t db = smem_desc_mn_major(sa + kStageBytesA);
+                    const uint64_t db = smem_desc_mn_major(sa + kPairStageBytesA);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma(tmem_acc, da + a_step * k, db + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    umma_commit(&bar.empty[stage]);
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        umma_pair(tmem_acc, da + a_step * k, db + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(&bar.empty[stage]);
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                 }
-                umma_commit(&bar.acc_full[acc]);
+                umma_commit_pair(&bar.acc_full[acc]);
                 if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -361,8 +379,8 @@ lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         int acc = 0;
         uint32_t acc_phase = 0;
-        for (int64_t tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
-            const int64_t row = (int64_t)(tile / g.n_tiles) * BM + row_in_tile;
+        for (int64_t tile = first; tile < n_tiles_total; tile += stride) {
+            const int64_t row = (int64_t)(tile / g.n_tiles) * 2 * BM + (int64_t)rank * BM + row_in_tile;
             const int n0 = (int)(tile % g.n_tiles) * BN;
             const bool row_ok = row < g.m_valid;
             float* const c_row = g.C + (row_ok ? row : 0) * g.ldc;
@@ -390,12 +408,12 @@ lm_head_grad_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.acc_empty[acc]);
+            if (lane == 0) mbar_arrive_leader(&bar.acc_empty[acc]);
             if (++acc == kAccumulators) { acc = 0; acc_phase ^= 1u; }
         }
     }
     if (timed_out && lane == 0) pods_raise(g.status, PODS_STATUS_TIMEOUT);
-    pipeline_teardown(tmem_base, warp);
+    pair_teardown(tmem_base, warp);
 }
 
 // How a call is cut up: the statistics plan, the panels of the vocabulary and the workspace regions.
@@ -404,17 +422,19 @@ struct Layout {
     int64_t rows_padded;         // T rounded up to whole 128-row blocks
     int total_tiles;             // 256-column tiles of the vocabulary
     int tiles_per_panel, n_panels;
-    int64_t ldp;                 // panel row pitch in elements = tiles_per_panel * 256
+    int64_t ldp;                 // panel row pitch in elements = tiles_per_panel * 256 + 64
     size_t off_row_loss, off_grad, off_panel, bytes;
 };
 
-// Time of one panel of c column tiles in units of one 128 x 256 x 64 block of tensor-core work: every kernel runs
-// its tiles in waves over the SMs, so what counts is (waves) x (contraction blocks per tile) for the three of them.
+// Time of one panel of c column tiles in units of one 128 x 256 x 64 block of tensor-core work per CTA: every kernel
+// runs its 256 x 256 pair tiles in waves over the SM pairs, so what counts is (waves) x (contraction blocks per tile)
+// for the three of them.
 int64_t panel_cost(int64_t c, int64_t row_blocks, int64_t d, int sms) {
+    const int64_t pairs = sms / 2 > 0 ? sms / 2 : 1, row_pairs = (row_blocks + 1) / 2;
     const int64_t n_d = (d + BN - 1) / BN;
-    const int64_t dlogits = (c * row_blocks + sms - 1) / sms * ((d + BK - 1) / BK);
-    const int64_t dhidden = (row_blocks * n_d + sms - 1) / sms * (c * BN / BK);
-    const int64_t dw = (2 * c * n_d + sms - 1) / sms * (row_blocks * BM / BK);
+    const int64_t dlogits = (c * row_pairs + pairs - 1) / pairs * ((d + BK - 1) / BK);
+    const int64_t dhidden = (row_pairs * n_d + pairs - 1) / pairs * (c * BN / BK);
+    const int64_t dw = (c * n_d + pairs - 1) / pairs * (row_blocks * BM / BK);
     return dlogits + dhidden + dw + 150;             // + three launches' ramp-up and tail
 }
 
@@ -436,7 +456,7 @@ Layout make_layout(int64_t T, int32_t V, int32_t d, int sms) {
         if (best < 0 || cost < best) { best = cost; l.tiles_per_panel = (int)c; }
     }
     l.n_panels = (l.total_tiles + l.tiles_per_panel - 1) / l.tiles_per_panel;
-    l.ldp = (int64_t)l.tiles_per_panel * BN;
+    l.ldp = (int64_t)l.tiles_per_panel * BN + 64;       // + one 128-byte line: rows of the panel must not be a power of two apart
     size_t off = align_up((size_t)l.stats.n_parts * (size_t)l.rows_padded * sizeof(float2), 256);
     l.off_row_loss = off;
     off += align_up((size_t)T * sizeof(double), 256);
@@ -450,10 +470,12 @@ Layout make_layout(int64_t T, int32_t V, int32_t d, int sms) {
 
 template <bool A_MN>
 int launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmArgs& g, int sms, cudaStream_t s) {
-    const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
-    if (tiles <= 0 || g.k_blocks <= 0) return PODS_OK;
-    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_grad_gemm_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    lm_head_grad_gemm_kernel<A_MN><<<(int)(tiles < sms ? tiles : sms), kThreads, kSmemBytes, s>>>(map_a, map_b, g);
+    if ((int64_t)g.m_tiles * g.n_tiles <= 0 || g.k_blocks <= 0) return PODS_OK;
+    // an even grid: one pair of CTAs per 256 x 256 tile at a time
+    const int64_t pair_tiles = (int64_t)((g.m_tiles + 1) / 2) * g.n_tiles;
+    const int64_t pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
+    PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_grad_gemm_pair_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
+    lm_head_grad_gemm_pair_kernel<A_MN><<<(int)(2 * pairs), kThreads, kPairSmemBytes, s>>>(map_a, map_b, g);
     PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
     return PODS_OK;
 }
@@ -554,12 +576,12 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
     CUtensorMap map_panel_rows, map_panel_box;   // the panel as K-major A (dhidden) and as MN-major A (dW)
     CUtensorMap map_panel_store;                 // the panel in 32 x 64 boxes: what an epilogue warp stores at a time
     if ((rc = make_map(&map_h_rows, hidden, T, d, ldh, BM)) != PODS_OK) return rc;
-    if ((rc = make_map(&map_w_rows, W, V, d, ldw, BN)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_w_rows, W, V, d, ldw, BN / 2)) != PODS_OK) return rc;
     if ((rc = make_map(&map_w_box, W, V, d, ldw, 64)) != PODS_OK) return rc;
     if ((rc = make_map(&map_h_box, hidden, T, d, ldh, 64)) != PODS_OK) return rc;
-    if ((rc = make_map(&map_panel_rows, panel, l.rows_padded, l.ldp, l.ldp, BM)) != PODS_OK) return rc;
-    if ((rc = make_map(&map_panel_box, panel, l.rows_padded, l.ldp, l.ldp, 64)) != PODS_OK) return rc;
-    if ((rc = make_map(&map_panel_store, panel, l.rows_padded, l.ldp, l.ldp, 32)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_panel_rows, panel, l.rows_padded, (int64_t)l.tiles_per_panel * BN, l.ldp, BM)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_panel_box, panel, l.rows_padded, (int64_t)l.tiles_per_panel * BN, l.ldp, 64)) != PODS_OK) return rc;
+    if ((rc = make_map(&map_panel_store, panel, l.rows_padded, (int64_t)l.tiles_per_panel * BN, l.ldp, 32)) != PODS_OK) return rc;
     PODS_RETURN_IF_CUDA_ERROR(cudaFuncSetAttribute(lm_head_dlogits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDlogitsSmemBytes));
 
     for (int p = 0; p < l.n_panels; ++p) {
@@ -572,15 +594,16 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
         DlogitsArgs da;
         da.V = V;
         da.d = d;
-        da.n_row_blocks = pp.n_row_blocks;
+        da.n_row_blocks = (pp.n_row_blocks + 1) / 2;
+        da.n_blocks128 = pp.n_row_blocks;
         da.tile0 = tile0;
         da.n_col_tiles = n_tiles;
-        da.group_rows = pp.n_row_blocks < 16 ? pp.n_row_blocks : 16;
-        da.n_items = (int64_t)n_tiles * pp.n_row_blocks;
+        da.group_rows = da.n_row_blocks < 8 ? da.n_row_blocks : 8;      // 8 pairs = 16 blocks of 128 rows
+        da.n_items = (int64_t)n_tiles * da.n_row_blocks;
         da.grad = grad;
         da.ldp = l.ldp;
         da.status = status;
-        lm_head_dlogits_kernel<<<(int)(da.n_items < sms ? da.n_items : sms), kDlogitsThreads, kDlogitsSmemBytes, s>>>(map_h_rows, map_w_rows, map_panel_store, da);
+        lm_head_dlogits_kernel<<<(int)(2 * (da.n_items < sms / 2 ? da.n_items : sms / 2)), kDlogitsThreads, kDlogitsSmemBytes, s>>>(map_h_rows, map_w_rows, map_panel_store, da);
         PODS_RETURN_IF_CUDA_ERROR(cudaGetLastError());
 
         GemmArgs gh;                             // dhidden[T, d] (+)= panel[T, cols] . W[tile0 * 256 + (0 .. cols), d]
