@@ -459,8 +459,8 @@ def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0, compare=True)
     flop_useful, flop_issued = 6.0 * T * V * d, 8.0 * T * V * d
     peaks = measured_peaks()
     burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
-    out = {"kernels": ["lm_head_stats_kernel", "lm_head_dlogits_kernel", "lm_head_grad_gemm_kernel<0>",
-                       "lm_head_grad_gemm_kernel<1>"], "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
+    out = {"kernels": ["lm_head_stats_kernel", "lm_head_dlogits_kernel", "lm_head_grad_gemm_pair_kernel<0>",
+                       "lm_head_grad_gemm_pair_kernel<1>"], "T": T, "V": V, "d": d, "bound": "tensor", "unit": "TFLOP/s",
            "ms_alone_best": min(alone), "ms_alone_all": alone,
            "issued_alone": flop_issued / min(alone) / 1e9, "useful_alone": flop_useful / min(alone) / 1e9,
            "peak_burst": burst, "frac_issued_alone_of_burst": flop_issued / min(alone) / 1e9 / burst,
@@ -470,6 +470,7 @@ def time_lm_head_loss(dev, T=16384, V=151936, d=2048, seconds=2.0, compare=True)
            "frac_useful_loop_of_sustained": flop_useful / ms_loop / 1e9 / sustained,
            "peak_kind": "of measured" if peaks else "of fallback",
            "sm_mhz_median": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
+           "ms_x_mhz_loop": ms_loop * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
            "tokens_per_s_loop": T / (ms_loop * 1e-3), "workspace_bytes": fused_bytes,
            "device_status_word": status_word}
     if not compare:
