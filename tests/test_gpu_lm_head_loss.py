@@ -180,6 +180,39 @@ def test_without_kl_strided_inputs_and_token_range():
     assert np.abs(bad["logp"] - want0["logp"]).max() <= LOGP_ATOL
 
 
+def test_chunks_with_row0_add_up_to_the_whole_batch():
+    """Two calls over rows [0, a) and [a, T) with the batch-wide cu_seqlens, weights and advantages (row0 = the chunk's
+    first packed row; the cut falls inside a rollout and off the 128-row grid), loss_acc and dW carried from one
+    call to the next: the same objective and gradients as one call over all rows."""
+    c = _inputs(700, 3000, 128, 5, seed=26, masked=(3, 400))
+    want = _oracle(c)
+    whole = _run(c)
+    dev = c["hidden"].device
+    a = 333
+    cu = torch.from_numpy(c["cu"]).to(dev)
+    mask = torch.from_numpy(c["mask"]).to(dev)
+    sw = binding.grpo_seq_weights(mask, cu)
+    loss_acc = torch.zeros(1, dtype=torch.float64, device=dev)
+    dW = torch.zeros((c["V"], c["d"]), dtype=torch.float32, device=dev)
+    status = binding.new_status()
+    old, ref, adv = (torch.from_numpy(c[k]).to(dev) for k in ("old", "ref", "adv"))
+    logps, dhs = [], []
+    for lo, hi in ((0, a), (a, c["T"])):
+        lp, dh = binding.grpo_loss_from_hidden(c["hidden"][lo:hi], c["W"], c["tokens"][lo:hi].contiguous(),
+                                               old[lo:hi].contiguous(), ref[lo:hi].contiguous(), adv, sw, cu, lo,
+                                               mask[lo:hi].contiguous(), EPS, BETA, loss_acc, dW, status=status)
+        logps.append(lp)
+        dhs.append(dh)
+    torch.cuda.synchronize()
+    got = dict(logp=torch.cat(logps).cpu().numpy(), dhidden=torch.cat(dhs).cpu().numpy().astype(np.float64),
+               dW=dW.cpu().numpy().astype(np.float64), loss=float(loss_acc.item()), status=binding.read_status(status))
+    _compare("grpo_loss_from_hidden two chunks", got, want, c)
+    assert got["logp"].tobytes() == whole["logp"].tobytes()
+    assert got["dhidden"].tobytes() == whole["dhidden"].tobytes()      # a row's results do not depend on its tile mates
+    assert abs(got["loss"] - whole["loss"]) <= 1e-12 * abs(whole["loss"]) + 1e-18
+    assert np.abs(got["dW"] - whole["dW"]).max() <= 1e-5 * np.abs(want["abs_dW"]).max()
+
+
 def test_repeated_calls_give_the_same_bits():
     c = _inputs(384, 5000, 192, 5, seed=24)
     a, b = _run(c), _run(c)
