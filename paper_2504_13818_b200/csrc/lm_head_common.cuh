@@ -227,6 +227,20 @@ __device__ __forceinline__ uint32_t leader_addr(const void* p) {
 __device__ __forceinline__ void mbar_arrive_leader(const void* bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_addr(bar)) : "memory");
 }
+// Bounded wait on one of this CTA's barriers whose arrivals come from BOTH CTAs of the pair: acquire at cluster scope.
+__device__ __forceinline__ bool mbar_wait_cluster(void* bar, uint32_t parity, bool hurry) {
+    const uint32_t limit = hurry ? 1u : kWaitLimit;
+    for (uint32_t i = 0; i < limit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, 1000;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok != 0) return true;
+    }
+    return false;
+}
 // A box into THIS CTA's shared memory; the bytes are counted on the LEADER's barrier at the same offset.
 __device__ __forceinline__ void tma_load_tile_pair(void* dst, const CUtensorMap* map, int x, int y, const void* bar) {
     asm volatile(

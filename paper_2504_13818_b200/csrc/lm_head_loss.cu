@@ -180,7 +180,7 @@ lm_head_dlogits_kernel(const __grid_constant__ CUtensorMap map_hidden, const __g
             uint32_t acc_phase = 0;
             for (int64_t item = first; item < a.n_items; item += stride) {
                 {
-                    if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
+                    if (!mbar_wait_cluster(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
                     tcgen05_fence_after();
                     const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
                     for (int kb = 0; kb < k_blocks; ++kb) {
@@ -353,7 +353,7 @@ lm_head_grad_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
             constexpr uint64_t a_step = A_MN ? (uint64_t)(UMMA_K * 128 >> 4) : (uint64_t)(UMMA_K * 2 >> 4);
             constexpr uint64_t b_step = (uint64_t)(UMMA_K * 128 >> 4);
             for (int64_t tile = first; tile < n_tiles_total; tile += stride) {
-                if (!mbar_wait(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
+                if (!mbar_wait_cluster(&bar.acc_empty[acc], acc_phase ^ 1u, timed_out)) timed_out = true;
                 tcgen05_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < g.k_blocks; ++kb) {
