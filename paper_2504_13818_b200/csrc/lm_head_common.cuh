@@ -70,14 +70,9 @@ __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map,
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
-// The same with an L2 eviction policy for the lines the load brings in.
-__device__ __forceinline__ void tma_load_tile_hint(void* dst, const CUtensorMap* map, int x, int y, void* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
-}
-// L2 policy for data that streams through once: first in line for eviction, so that it does not push out the
-// matrices every CTA keeps re-reading.
+// L2 policy for data that is written once and read much later (the gradient panel's stores): first in line for
+// eviction.  NOT for loads that several CTAs share: with this hint on the panel's loads the sharers' later requests
+// missed and the panel crossed HBM three to four times.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
@@ -246,12 +241,6 @@ __device__ __forceinline__ void tma_load_tile_pair(void* dst, const CUtensorMap*
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(leader_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void tma_load_tile_pair_hint(void* dst, const CUtensorMap* map, int x, int y, const void* bar,
-                                                        uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(leader_addr(bar)), "l"(policy) : "memory");
 }
 // Instruction descriptor of the pair's MMA: M = 256 (128 rows in each CTA), N = 256.
 __host__ __device__ constexpr uint32_t instr_desc_pair(bool a_mn_major, bool b_mn_major) {

@@ -103,8 +103,9 @@ struct DlogitsArgs {
 
 // Order of the panel's tiles: groups of `group_rows` blocks of rows; inside a group one column tile after the other,
 // and for each the group's row blocks.  The CTAs that run at the same time (consecutive items) then share a few
-// column tiles of W and a few row blocks of hidden - 17 MB at 16 row blocks per group - instead of sweeping all of
-// hidden (67 MB at 16384 rows, more than one L2 partition holds) for every column tile.
+// column tiles of W and the group's row blocks of hidden - 32 MB at 64 row blocks per group and d = 2048 - instead of
+// sweeping all of hidden (67 MB at 16384 rows, more than one L2 partition holds) for every column tile, and the
+// panel's rows of W cross HBM once per group (2 to 4 times per panel; 8 times with groups of 16 row blocks).
 __device__ __forceinline__ void tile_of(const DlogitsArgs& a, int64_t item, int* ct, int* rb) {
     const int64_t per_group = (int64_t)a.group_rows * a.n_col_tiles;
     const int n_groups = (a.n_row_blocks + a.group_rows - 1) / a.group_rows;
@@ -318,7 +319,6 @@ lm_head_grad_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
             int stage = 0;
             uint32_t phase = 0;
             int64_t loads = 0;
-            const uint64_t stream_policy = l2_policy_evict_first();
             for (int64_t tile = first; tile < n_tiles_total; tile += stride) {
                 const int m0 = (int)(tile / g.n_tiles) * 2 * BM + (int)rank * BM;
                 const int n0 = (int)(tile % g.n_tiles) * BN + (int)rank * (BN / 2);
@@ -329,9 +329,9 @@ lm_head_grad_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
                     if (A_MN) {
 #pragma unroll
                         for (int i = 0; i < BM / 64; ++i)
-                            tma_load_tile_pair_hint(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage], stream_policy);
+                            tma_load_tile_pair(sa + i * kBoxBytes, &map_a, m0 + 64 * i, kb * BK, &bar.full[stage]);
                     } else {
-                        tma_load_tile_pair_hint(sa, &map_a, kb * BK, m0, &bar.full[stage], stream_policy);
+                        tma_load_tile_pair(sa, &map_a, kb * BK, m0, &bar.full[stage]);
                     }
 #pragma unroll
                     for (int i = 0; i < BN / 2 / 64; ++i)
@@ -598,7 +598,7 @@ extern "C" int grpo_loss_from_hidden(const void* hidden, int64_t ldh, const void
         da.n_blocks128 = pp.n_row_blocks;
         da.tile0 = tile0;
         da.n_col_tiles = n_tiles;
-        da.group_rows = da.n_row_blocks < 8 ? da.n_row_blocks : 8;      // 8 pairs = 16 blocks of 128 rows
+        da.group_rows = da.n_row_blocks < 32 ? da.n_row_blocks : 32;    // 32 pairs = 64 blocks of 128 rows
         da.n_items = (int64_t)n_tiles * da.n_row_blocks;
         da.grad = grad;
         da.ldp = l.ldp;
